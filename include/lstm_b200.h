@@ -1,0 +1,159 @@
+/*
+ * lstm_b200 -- stacked (optionally bidirectional) LSTM inference forward pass on one sm_100a GPU.
+ *
+ * C ABI: plain pointers and sizes only.  Every function returns one of the LSTM_* codes below (except
+ * lstm_last_error); on failure lstm_last_error(handle) -- or lstm_last_error(NULL) for a failed
+ * lstm_create -- returns a human-readable reason.  No function falls back to the CPU: without a usable
+ * CUDA device every call fails with LSTM_ERR_CUDA.
+ *
+ * What is computed (paper, Section 4, the cell-equation block, with zero hidden layers inside each
+ * gate, i.e. the conventional LSTM the paper takes as its baseline in Sections 5.1 and 5.2).  For
+ * layer l, direction d, timestep t in processing order (forward 0..T-1; reverse T-1..0), batch row b,
+ * hidden unit j, with W = [Wx | Wh] acting on the concatenation [x_t, h_{t-1}]:
+ *
+ *     z_q[j] = b_q[j] + sum_k Wx_q[j,k] X_l[t,b,k] + sum_k Wh_q[j,k] h_prev[b,k]     q in {i,f,g,o}
+ *     i = sigmoid(z_i)  f = sigmoid(z_f)  g = tanh(z_g)  o = sigmoid(z_o)
+ *     c = f * c_prev + i * g             h = o * tanh(c)
+ *
+ * X_0 = x; X_l for l > 0 is the previous layer's output [T,B,D*H] (forward half first, then reverse).
+ * Pruned weights follow the mask-based scheme of Section 4: the effective matrix is W (x) Msk.
+ *
+ * Layout conventions
+ *   - Gate rows are packed in four blocks of H rows in the order i, f, g, o: row q*H + j.
+ *   - All activations are fp32, contiguous, time-major: x [T,B,in_dim], y [T,B,D*H].
+ *   - State tensors are [L*D, B, H]; entry l*D + d (d = 1 is the reverse direction).  The reverse
+ *     direction starts from h0/c0[l*D+1] at t = T-1 and its final state is the one after t = 0.
+ *   - A handle is bound to the device that was current in lstm_create; calls on one handle must not
+ *     overlap (one handle is not thread-safe); different handles are independent.
+ */
+#ifndef LSTM_B200_H
+#define LSTM_B200_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LSTM_API __attribute__((visibility("default")))
+#else
+#define LSTM_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lstm_handle lstm_handle;      /* opaque, library-owned */
+
+/* storage / arithmetic type */
+enum {
+    LSTM_F32       = 0,   /* fp32 weights, fp32 activations and state, fp32 accumulation              */
+    LSTM_BF16W_F32S = 1   /* weights rounded to bf16 (nearest-even) at create time; the input
+                             projection also rounds its activations to bf16 (tensor-core operands);
+                             state, accumulation, gates and outputs are fp32                            */
+};
+
+/* return codes */
+enum {
+    LSTM_OK = 0,
+    LSTM_ERR_INVALID = 1,      /* bad argument (NULL, shape, T > max_T, malformed CSR ...); nothing launched */
+    LSTM_ERR_UNSUPPORTED = 2,  /* valid request the library cannot serve (e.g. hidden >= 65536)            */
+    LSTM_ERR_CUDA = 3,         /* a CUDA call failed (no device, launch refused ...)                        */
+    LSTM_ERR_NOMEM = 4,        /* host or device allocation failed                                           */
+    LSTM_ERR_TIMEOUT = 5       /* a device-side wait of the recurrent kernel gave up; outputs undefined     */
+};
+
+/* how the recurrent and input matrices are executed */
+enum {
+    LSTM_DENSE = 0,   /* dense kernels; a mask, if given, is applied as explicit zeros                 */
+    LSTM_CSR   = 1    /* sparse kernels over the surviving entries only (from masks or caller CSR)      */
+};
+
+/*
+ * Weights of one (layer, direction); array index = layer*D + direction.  All pointers may be host or
+ * device pointers (the library finds out which) and are only read during lstm_create; the caller may
+ * free them afterwards.
+ *   dense form:  wx [4H, in_l], wh [4H, H] row-major fp32 (in_l = in_dim for layer 0, D*H after);
+ *                optional masks of the same shapes, uint8, 1 = keep (the paper's Msk), NULL = keep all.
+ *   CSR form:    used for a matrix when its rowptr is non-NULL (then the dense pointer and mask of
+ *                that matrix are ignored): rowptr int32[4H+1] starting at 0, col int32[nnz] strictly
+ *                increasing inside each row and within range, val fp32[nnz].
+ *   b:           [4H] single bias per gate (a two-bias convention passes the sum); NULL = zeros.
+ */
+typedef struct {
+    const float   *wx;
+    const float   *wh;
+    const float   *b;
+    const uint8_t *mask_x;
+    const uint8_t *mask_h;
+    const int32_t *wx_rowptr; const int32_t *wx_col; const float *wx_val;
+    const int32_t *wh_rowptr; const int32_t *wh_col; const float *wh_val;
+} lstm_weights;
+
+/*
+ * Create-time packing (Section 4: W <- W (x) Msk once training has finished; here: once, at create).
+ * Copies, masks, rounds (bf16 mode) and re-tiles all weights into library-owned device memory, and
+ * allocates the workspace for sequences up to max_T steps and max_B batch rows.
+ *   layers >= 1, in_dim >= 1, 1 <= hidden < 65536, bidir in {0,1}, dtype LSTM_F32 | LSTM_BF16W_F32S,
+ *   w[layers*(1+bidir)], exec_mode LSTM_DENSE | LSTM_CSR, 1 <= max_T, 1 <= max_B,
+ *   cuda_stream: a cudaStream_t (NULL = default stream) used for the uploads.
+ * Synchronises the stream before returning.  On failure *out is NULL.
+ */
+LSTM_API int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir, int dtype,
+                const lstm_weights *w, int exec_mode, int max_T, int max_B, void *cuda_stream);
+
+/*
+ * Forward pass over a whole sequence batch; all pointers are DEVICE pointers owned by the caller.
+ *   x  [T,B,in_dim]      h0, c0 [L*D,B,H] or NULL (zeros)
+ *   y  [T,B,D*H]         hT, cT [L*D,B,H] or NULL (not wanted)
+ * 0 <= T <= max_T, 0 <= B <= max_B (T = 0 or B = 0: nothing is launched; hT,cT receive h0,c0).
+ * Work is enqueued on cuda_stream and the call returns without synchronising; a device-side timeout
+ * of this call is reported by the next lstm_forward / lstm_status on the handle.
+ * Steps, in order, per layer: input staging (bf16 mode), input projection for all timesteps at once
+ * (the x_t half of W [x_t, h_{t-1}] + b), then the serial recurrence with the gate nonlinearities and
+ * the c/h update fused into one persistent kernel.
+ */
+LSTM_API int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, const float *c0,
+                 float *y, float *hT, float *cT, void *cuda_stream);
+
+/*
+ * Same computation with HOST buffers (pinned or pageable): copies x (and h0, c0 if given) to
+ * handle-owned device staging buffers, runs lstm_forward, copies y (and hT, cT if wanted) back, and
+ * synchronises cuda_stream before returning, so the device status of this very call is returned.
+ */
+LSTM_API int lstm_forward_host(lstm_handle *h, const float *x, int T, int B, const float *h0, const float *c0,
+                      float *y, float *hT, float *cT, void *cuda_stream);
+
+/* Synchronises the stream last used with the handle and returns LSTM_OK or the recorded device
+ * status (LSTM_ERR_TIMEOUT ...); the recorded status is cleared. */
+LSTM_API int lstm_status(lstm_handle *h);
+
+/* Frees everything the handle owns (synchronises the device first).  NULL is accepted. */
+LSTM_API int lstm_destroy(lstm_handle *h);
+
+/* Reason of the last failure on this handle (or of the last failed lstm_create when h is NULL).
+ * The string is owned by the library and valid until the next failing call. */
+LSTM_API const char *lstm_last_error(const lstm_handle *h);
+
+/*
+ * Measurement support.  With profiling on, lstm_forward brackets each of its kernels with CUDA events
+ * on the launching stream; lstm_profile_read synchronises and returns, for the most recent
+ * lstm_forward, per kernel kind k (LSTM_K_*): launches[k] and total device milliseconds ms[k].
+ * Arrays must have LSTM_K_COUNT entries.
+ */
+enum { LSTM_K_STAGE = 0, LSTM_K_PROJ = 1, LSTM_K_RECUR = 2, LSTM_K_COUNT = 3 };
+LSTM_API int lstm_profile_enable(lstm_handle *h, int on);
+LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
+
+/*
+ * Read-only facts about how the handle runs (for reports): writes up to n values into out and
+ * returns the number available.  Order: [0] SM count, [1] CTAs of the recurrent kernel per direction,
+ * [2] threads per CTA, [3] dynamic shared memory bytes per CTA at max_B, [4] recurrent-matrix rows
+ * resident in shared memory per CTA (max over CTAs), [5] rows streamed from L2 per CTA (max),
+ * [6] split-K factor of the input projection at max_T*max_B, [7] 1 if the projection uses the tensor-core
+ * (tcgen05) kernel, [8] kernels launched by one lstm_forward at (max_T, max_B).
+ */
+LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LSTM_B200_H */

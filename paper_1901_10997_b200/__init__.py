@@ -1,0 +1,12 @@
+"""Stacked-LSTM inference forward pass on one B200 (sm_100a): thin Python binding of liblstm_b200.so.
+
+Every step of the computation runs in the library's CUDA kernels; this package only marshals
+arguments.  There is no CPU fallback: if the shared library is missing or no CUDA device is usable,
+the calls raise.
+"""
+from .binding import (LSTM, LstmError, lib_path, load_library, lstm_create, lstm_destroy,  # noqa: F401
+                      lstm_forward, lstm_forward_host, lstm_info, lstm_last_error,
+                      lstm_profile_enable, lstm_profile_read, lstm_status,
+                      LSTM_F32, LSTM_BF16W_F32S, LSTM_DENSE, LSTM_CSR, LSTM_OK, LSTM_ERR_INVALID,
+                      LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT,
+                      LSTM_K_STAGE, LSTM_K_PROJ, LSTM_K_RECUR, LSTM_K_COUNT)

@@ -1,0 +1,723 @@
+// C ABI of the lstm_b200 library: create-time packing, the per-layer launch sequence, host-buffer
+// variant, status and measurement support.  See include/lstm_b200.h for the contract.
+#include "../../include/lstm_b200.h"
+#include "common.cuh"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace lstm;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct Layer {
+    int in_l = 0;
+    int ldk = 0;                       // row stride of wx (elements)
+    void *wx = nullptr;                // dense [D*4H][ldk], rows in order d*4H + j*4 + q
+    float *bias = nullptr;             // [D*4H], same order
+    int *wx_rowptr = nullptr;          // CSR projection [D*4H + 1]
+    CsrEntry *wx_ent = nullptr;
+    void *wh[2] = {nullptr, nullptr};  // dense [H][4][Hp8]
+    int *wh_ptr[2] = {nullptr, nullptr};   // CSR recurrence: padded entry offsets [4H+1]
+    void *wh_ent[2] = {nullptr, nullptr};
+    int csr_max_slice_entries = 0;     // largest per-CTA slice (entries, padded)
+    ProjTcPlan plan;                   // tensor-core projection plan for plan_M rows
+    int plan_M = -1;
+};
+
+}  // namespace
+
+struct lstm_handle {
+    int L = 0, D = 1, in_dim = 0, H = 0, dtype = 0, exec_mode = 0, max_T = 0, max_B = 0;
+    int device = 0, sm_count = 0, smem_optin = 0;
+    int Hp8 = 0, Hs = 0;
+    int ncta_dir = 0, upc = 0, threads = 0;
+    bool use_tc = false;
+    std::vector<Layer> layers;
+    // workspace
+    float *G = nullptr; size_t G_cap = 0;
+    __nv_bfloat16 *xb0 = nullptr; int ld0 = 0;
+    __nv_bfloat16 *xbn[2] = {nullptr, nullptr}; int ldn = 0;
+    float *ybuf[2] = {nullptr, nullptr};
+    unsigned long long *xch = nullptr; size_t xch_words = 0;
+    int *status_dev = nullptr;
+    unsigned stamp_next = 0;
+    long long spin_limit = 2000000000LL;
+    cudaStream_t last_stream = nullptr;
+    // host-buffer variant staging
+    float *hx = nullptr, *hy = nullptr, *hh0 = nullptr, *hc0 = nullptr, *hhT = nullptr, *hcT = nullptr;
+    // profiling
+    bool prof = false;
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> ev_kind;
+    int ev_used = 0;
+    int last_launches = 0;
+    std::string err;
+};
+
+namespace {
+
+int fail(lstm_handle *h, int code, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (h) h->err = buf; else g_create_error = buf;
+    return code;
+}
+
+inline uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);   // NaN stays NaN
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+inline float bf16_to_f32(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+// Returns a host-readable view of n bytes at p (copying from the device when p is device memory).
+struct HostView {
+    std::vector<unsigned char> copy;
+    const void *ptr = nullptr;
+};
+bool host_view(const void *p, size_t bytes, HostView &v)
+{
+    v.ptr = p;
+    if (!p || bytes == 0) return true;
+    cudaPointerAttributes at;
+    cudaError_t e = cudaPointerGetAttributes(&at, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return true; }      // plain host memory on old drivers
+    if (at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged) {
+        v.copy.resize(bytes);
+        if (cudaMemcpy(v.copy.data(), p, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return false;
+        v.ptr = v.copy.data();
+    }
+    return true;
+}
+
+// One matrix in row-compressed host form: kept entries of each row in increasing column order.
+struct HostCsr {
+    std::vector<int> rowptr;
+    std::vector<int> col;
+    std::vector<float> val;
+};
+
+// Normalises either description of a [rows x cols] matrix into HostCsr (keep_zeros: with a mask, a
+// kept entry whose value is 0 stays an entry; without mask or CSR, only non-zero values are kept).
+int matrix_to_csr(lstm_handle *h, int rows, int cols, const float *dense, const uint8_t *mask,
+                  const int32_t *rowptr, const int32_t *col, const float *val, HostCsr &out, const char *name)
+{
+    out.rowptr.assign(rows + 1, 0);
+    if (rowptr) {
+        HostView rp, cv, vv;
+        if (!host_view(rowptr, sizeof(int32_t) * (rows + 1), rp)) return fail(h, LSTM_ERR_CUDA, "reading %s rowptr", name);
+        const int32_t *r = (const int32_t *)rp.ptr;
+        if (r[0] != 0) return fail(h, LSTM_ERR_INVALID, "%s: CSR rowptr[0] != 0", name);
+        for (int i = 0; i < rows; ++i)
+            if (r[i + 1] < r[i]) return fail(h, LSTM_ERR_INVALID, "%s: CSR rowptr decreases at row %d", name, i);
+        const int nnz = r[rows];
+        if (nnz > 0 && (!col || !val)) return fail(h, LSTM_ERR_INVALID, "%s: CSR col/val missing", name);
+        if (!host_view(col, sizeof(int32_t) * nnz, cv) || !host_view(val, sizeof(float) * nnz, vv))
+            return fail(h, LSTM_ERR_CUDA, "reading %s CSR arrays", name);
+        const int32_t *c = (const int32_t *)cv.ptr;
+        const float *v = (const float *)vv.ptr;
+        for (int i = 0; i < rows; ++i)
+            for (int e = r[i]; e < r[i + 1]; ++e) {
+                if (c[e] < 0 || c[e] >= cols) return fail(h, LSTM_ERR_INVALID, "%s: CSR column %d out of range in row %d", name, c[e], i);
+                if (e > r[i] && c[e] <= c[e - 1]) return fail(h, LSTM_ERR_INVALID, "%s: CSR columns not strictly increasing in row %d", name, i);
+            }
+        out.rowptr.assign(r, r + rows + 1);
+        out.col.assign(c, c + nnz);
+        out.val.assign(v, v + nnz);
+        return LSTM_OK;
+    }
+    if (!dense) return fail(h, LSTM_ERR_INVALID, "%s: neither dense nor CSR weights given", name);
+    HostView dv, mv;
+    if (!host_view(dense, sizeof(float) * (size_t)rows * cols, dv) || !host_view(mask, (size_t)rows * cols, mv))
+        return fail(h, LSTM_ERR_CUDA, "reading %s", name);
+    const float *w = (const float *)dv.ptr;
+    const uint8_t *m = (const uint8_t *)mv.ptr;
+    for (int i = 0; i < rows; ++i) {
+        for (int k = 0; k < cols; ++k) {
+            const size_t idx = (size_t)i * cols + k;
+            const bool keep = m ? (m[idx] != 0) : (w[idx] != 0.0f);
+            if (keep) { out.col.push_back(k); out.val.push_back(w[idx]); }
+        }
+        out.rowptr[i + 1] = (int)out.col.size();
+    }
+    return LSTM_OK;
+}
+
+// Dense [rows x cols] fp32 with the mask applied as explicit zeros (W (x) Msk), from either form.
+int matrix_to_dense(lstm_handle *h, int rows, int cols, const float *dense, const uint8_t *mask,
+                    const int32_t *rowptr, const int32_t *col, const float *val, std::vector<float> &out,
+                    const char *name)
+{
+    out.assign((size_t)rows * cols, 0.0f);
+    if (rowptr) {
+        HostCsr c;
+        int rc = matrix_to_csr(h, rows, cols, nullptr, nullptr, rowptr, col, val, c, name);
+        if (rc) return rc;
+        for (int i = 0; i < rows; ++i)
+            for (int e = c.rowptr[i]; e < c.rowptr[i + 1]; ++e) out[(size_t)i * cols + c.col[e]] = c.val[e];
+        return LSTM_OK;
+    }
+    if (!dense) return fail(h, LSTM_ERR_INVALID, "%s: neither dense nor CSR weights given", name);
+    HostView dv, mv;
+    if (!host_view(dense, sizeof(float) * (size_t)rows * cols, dv) || !host_view(mask, (size_t)rows * cols, mv))
+        return fail(h, LSTM_ERR_CUDA, "reading %s", name);
+    const float *w = (const float *)dv.ptr;
+    const uint8_t *m = (const uint8_t *)mv.ptr;
+    for (size_t i = 0; i < out.size(); ++i) out[i] = (m && !m[i]) ? 0.0f : w[i];
+    return LSTM_OK;
+}
+
+template <typename T>
+int upload(lstm_handle *h, T **dst, const void *src, size_t bytes, cudaStream_t st, const char *what)
+{
+    *dst = nullptr;
+    if (cudaMalloc((void **)dst, bytes ? bytes : 16) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(h, LSTM_ERR_NOMEM, "device allocation of %zu bytes for %s failed", bytes, what);
+    }
+    if (bytes && cudaMemcpyAsync(*dst, src, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return fail(h, LSTM_ERR_CUDA, "upload of %s failed: %s", what, cudaGetErrorString(cudaGetLastError()));
+    // the source vectors are pageable host memory: the async copy stages them before returning
+    return LSTM_OK;
+}
+
+template <typename T>
+int dev_alloc(lstm_handle *h, T **dst, size_t bytes, bool zero, cudaStream_t st, const char *what)
+{
+    *dst = nullptr;
+    if (cudaMalloc((void **)dst, bytes ? bytes : 16) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(h, LSTM_ERR_NOMEM, "device allocation of %zu bytes for %s failed", bytes, what);
+    }
+    if (zero && bytes && cudaMemsetAsync(*dst, 0, bytes, st) != cudaSuccess)
+        return fail(h, LSTM_ERR_CUDA, "clearing %s failed", what);
+    return LSTM_OK;
+}
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+void unit_range_host(int H, int nc, int c, int &u0, int &n)
+{
+    const int base = H / nc, rem = H % nc;
+    n = base + (c < rem ? 1 : 0);
+    u0 = c * base + std::min(c, rem);
+}
+
+// Launch shape of the recurrent kernel for B batch rows.
+struct RecurShape { int BT; size_t smem; int w_smem_bytes; int units_res_min; };
+
+RecurShape recur_shape(const lstm_handle *h, int B, int layer)
+{
+    const size_t budget = (size_t)h->smem_optin - 64;            // static shared memory of the kernel
+    const bool csr = h->exec_mode == LSTM_CSR;
+    const size_t wsize = h->dtype == LSTM_BF16W_F32S ? 2 : 4;
+    size_t need_w;
+    if (!csr) need_w = (size_t)h->upc * 4 * h->Hp8 * wsize;
+    else {
+        const size_t esize = h->dtype == LSTM_BF16W_F32S ? 4 : 8;
+        need_w = (size_t)round_up(4 * h->upc + 1, 4) * 4 + (size_t)h->layers[layer].csr_max_slice_entries * esize;
+    }
+    const size_t c_bytes = (size_t)round_up(h->upc * B, 4) * 4;
+    auto fixed = [&](int bt) { return (size_t)2 * bt * h->Hs * 4 + c_bytes; };
+    // candidates in order of preference: cost per weight ~ chunks * (1 unpack + BT FMAs)
+    int cands[4]; int nc = 0;
+    if (B <= 1) cands[nc++] = 1;
+    else if (B == 2) { cands[nc++] = 2; cands[nc++] = 1; }
+    else if (B <= 4) { cands[nc++] = 4; cands[nc++] = 2; cands[nc++] = 1; }
+    else if (h->dtype == LSTM_F32) { cands[nc++] = 4; cands[nc++] = 2; cands[nc++] = 1; }   // fp64 accumulators
+    else {
+        const int c8 = ((B + 7) / 8) * 9, c4 = ((B + 3) / 4) * 5;
+        if (c8 <= c4) { cands[nc++] = 8; cands[nc++] = 4; } else { cands[nc++] = 4; cands[nc++] = 8; }
+        cands[nc++] = 2; cands[nc++] = 1;
+    }
+    int pick = cands[nc - 1];
+    for (int i = 0; i < nc; ++i)
+        if (fixed(cands[i]) + need_w <= budget) { pick = cands[i]; break; }
+    RecurShape s;
+    s.BT = pick;
+    const size_t f = fixed(pick);
+    const size_t avail = budget > f ? budget - f : 0;
+    const size_t w = std::min(need_w, avail);
+    s.w_smem_bytes = (int)w;
+    s.smem = f + w;
+    s.units_res_min = 0;
+    return s;
+}
+
+int max_b_fits(const lstm_handle *h)
+{
+    // the staging buffers and the c state must fit even when no weight is resident
+    const size_t budget = (size_t)h->smem_optin - 64;
+    const size_t c_bytes = (size_t)round_up(h->upc * h->max_B, 4) * 4;
+    const size_t rp = h->exec_mode == LSTM_CSR ? (size_t)round_up(4 * h->upc + 1, 4) * 4 : 0;
+    return (size_t)2 * h->Hs * 4 + c_bytes + rp <= budget;
+}
+
+void free_all(lstm_handle *h)
+{
+    for (auto &ly : h->layers) {
+        cudaFree(ly.wx); cudaFree(ly.bias); cudaFree(ly.wx_rowptr); cudaFree(ly.wx_ent);
+        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); }
+    }
+    cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
+    cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->status_dev);
+    cudaFree(h->hx); cudaFree(h->hy); cudaFree(h->hh0); cudaFree(h->hc0); cudaFree(h->hhT); cudaFree(h->hcT);
+    for (auto e : h->ev) cudaEventDestroy(e);
+    cudaGetLastError();
+}
+
+bool want_tc(const lstm_handle *h)
+{
+    if (h->dtype != LSTM_BF16W_F32S || h->exec_mode != LSTM_DENSE) return false;
+    const char *env = getenv("LSTM_B200_PROJ");
+    return env && strcmp(env, "tc") == 0;
+}
+
+int n_split_cap() { return 4; }
+
+}  // namespace
+
+extern "C" {
+
+const char *lstm_last_error(const lstm_handle *h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir, int dtype,
+                const lstm_weights *w, int exec_mode, int max_T, int max_B, void *cuda_stream)
+{
+    if (!out) return fail(nullptr, LSTM_ERR_INVALID, "out is NULL");
+    *out = nullptr;
+    if (layers < 1 || in_dim < 1 || hidden < 1 || (bidir != 0 && bidir != 1) || !w || max_T < 1 || max_B < 1)
+        return fail(nullptr, LSTM_ERR_INVALID, "bad argument: layers=%d in_dim=%d hidden=%d bidir=%d max_T=%d max_B=%d w=%p",
+                    layers, in_dim, hidden, bidir, max_T, max_B, (const void *)w);
+    if (dtype != LSTM_F32 && dtype != LSTM_BF16W_F32S) return fail(nullptr, LSTM_ERR_INVALID, "unknown dtype %d", dtype);
+    if (exec_mode != LSTM_DENSE && exec_mode != LSTM_CSR) return fail(nullptr, LSTM_ERR_INVALID, "unknown exec_mode %d", exec_mode);
+    if (hidden >= 65536) return fail(nullptr, LSTM_ERR_UNSUPPORTED, "hidden must be < 65536");
+    if ((long long)max_T * max_B > (1LL << 30)) return fail(nullptr, LSTM_ERR_UNSUPPORTED, "max_T*max_B too large");
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        const char *m = cudaGetErrorString(cudaGetLastError());
+        return fail(nullptr, LSTM_ERR_CUDA, "no usable CUDA device: %s", m);
+    }
+    if (prop.major != 10) return fail(nullptr, LSTM_ERR_CUDA, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+    int coop = 0;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (!coop) return fail(nullptr, LSTM_ERR_CUDA, "device does not support cooperative launch");
+
+    lstm_handle *h = new (std::nothrow) lstm_handle;
+    if (!h) return fail(nullptr, LSTM_ERR_NOMEM, "host allocation failed");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    h->L = layers; h->D = bidir ? 2 : 1; h->in_dim = in_dim; h->H = hidden; h->dtype = dtype;
+    h->exec_mode = exec_mode; h->max_T = max_T; h->max_B = max_B; h->device = dev;
+    h->sm_count = prop.multiProcessorCount;
+    h->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    h->last_stream = st;
+    const int H = hidden, D = h->D;
+    const bool bf16 = dtype == LSTM_BF16W_F32S;
+    const bool csr = exec_mode == LSTM_CSR;
+    h->Hp8 = round_up(H, 8);
+    h->Hs = round_up(H, 256);
+    h->ncta_dir = std::max(1, std::min(h->sm_count / D, H));
+    h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
+    h->threads = std::max(128, 32 * std::min(h->upc, 16));
+    h->use_tc = want_tc(h);
+    h->layers.resize(layers);
+    if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
+
+    int rc = LSTM_OK;
+    auto bail = [&](int code) { g_create_error = h->err; free_all(h); delete h; return code; };
+    if (!max_b_fits(h)) { fail(h, LSTM_ERR_UNSUPPORTED, "hidden=%d with max_B=%d does not fit the recurrent kernel's shared memory", H, max_B); return bail(LSTM_ERR_UNSUPPORTED); }
+
+    for (int l = 0; l < layers && rc == LSTM_OK; ++l) {
+        Layer &ly = h->layers[l];
+        ly.in_l = l == 0 ? in_dim : D * H;
+        ly.ldk = bf16 ? round_up(ly.in_l, 8) : ly.in_l;
+        if (csr && (size_t)ly.in_l * 8 * 4 > (size_t)h->smem_optin) { rc = fail(h, LSTM_ERR_UNSUPPORTED, "sparse projection supports input widths up to %d", h->smem_optin / 32); break; }
+        const int N = D * 4 * H;
+        std::vector<float> bias_p((size_t)N, 0.0f);
+        std::vector<uint16_t> wx16; std::vector<float> wx32;
+        std::vector<int> px_rowptr; std::vector<CsrEntry> px_ent;
+        if (!csr) { if (bf16) wx16.assign((size_t)N * ly.ldk, 0); else wx32.assign((size_t)N * ly.ldk, 0.0f); }
+        else px_rowptr.assign(N + 1, 0);
+
+        for (int d = 0; d < D && rc == LSTM_OK; ++d) {
+            const lstm_weights &src = w[l * D + d];
+            char name[64];
+            // bias
+            if (src.b) {
+                HostView bv;
+                if (!host_view(src.b, sizeof(float) * 4 * H, bv)) { rc = fail(h, LSTM_ERR_CUDA, "reading bias"); break; }
+                const float *b = (const float *)bv.ptr;
+                for (int q = 0; q < 4; ++q)
+                    for (int j = 0; j < H; ++j) bias_p[(size_t)d * 4 * H + (size_t)j * 4 + q] = b[q * H + j];
+            }
+            if (!csr) {
+                std::vector<float> m;
+                snprintf(name, sizeof name, "wx[layer %d, dir %d]", l, d);
+                rc = matrix_to_dense(h, 4 * H, ly.in_l, src.wx, src.mask_x, src.wx_rowptr, src.wx_col, src.wx_val, m, name);
+                if (rc) break;
+                for (int q = 0; q < 4; ++q)
+                    for (int j = 0; j < H; ++j) {
+                        const float *srow = m.data() + (size_t)(q * H + j) * ly.in_l;
+                        const size_t drow = ((size_t)d * 4 * H + (size_t)j * 4 + q) * ly.ldk;
+                        if (bf16) for (int k = 0; k < ly.in_l; ++k) wx16[drow + k] = f32_to_bf16_rne(srow[k]);
+                        else memcpy(&wx32[drow], srow, sizeof(float) * ly.in_l);
+                    }
+                snprintf(name, sizeof name, "wh[layer %d, dir %d]", l, d);
+                rc = matrix_to_dense(h, 4 * H, H, src.wh, src.mask_h, src.wh_rowptr, src.wh_col, src.wh_val, m, name);
+                if (rc) break;
+                const size_t n = (size_t)H * 4 * h->Hp8;
+                if (bf16) {
+                    std::vector<uint16_t> p(n, 0);
+                    for (int j = 0; j < H; ++j)
+                        for (int q = 0; q < 4; ++q) {
+                            const float *srow = m.data() + (size_t)(q * H + j) * H;
+                            uint16_t *drow = p.data() + ((size_t)j * 4 + q) * h->Hp8;
+                            for (int k = 0; k < H; ++k) drow[k] = f32_to_bf16_rne(srow[k]);
+                        }
+                    rc = upload(h, &ly.wh[d], p.data(), n * 2, st, "recurrent weights");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                } else {
+                    std::vector<float> p(n, 0.0f);
+                    for (int j = 0; j < H; ++j)
+                        for (int q = 0; q < 4; ++q)
+                            memcpy(p.data() + ((size_t)j * 4 + q) * h->Hp8, m.data() + (size_t)(q * H + j) * H, sizeof(float) * H);
+                    rc = upload(h, &ly.wh[d], p.data(), n * 4, st, "recurrent weights");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                }
+            } else {
+                HostCsr cx, ch;
+                snprintf(name, sizeof name, "wx[layer %d, dir %d]", l, d);
+                rc = matrix_to_csr(h, 4 * H, ly.in_l, src.wx, src.mask_x, src.wx_rowptr, src.wx_col, src.wx_val, cx, name);
+                if (rc) break;
+                for (int j = 0; j < H; ++j)
+                    for (int q = 0; q < 4; ++q) {
+                        const int r = q * H + j;
+                        for (int e = cx.rowptr[r]; e < cx.rowptr[r + 1]; ++e) {
+                            float v = cx.val[e];
+                            if (bf16) v = bf16_to_f32(f32_to_bf16_rne(v));
+                            px_ent.push_back(CsrEntry{v, cx.col[e]});
+                        }
+                        px_rowptr[(size_t)d * 4 * H + (size_t)j * 4 + q + 1] = (int)px_ent.size();
+                    }
+                snprintf(name, sizeof name, "wh[layer %d, dir %d]", l, d);
+                rc = matrix_to_csr(h, 4 * H, H, src.wh, src.mask_h, src.wh_rowptr, src.wh_col, src.wh_val, ch, name);
+                if (rc) break;
+                std::vector<int> ptr(4 * H + 1, 0);
+                std::vector<unsigned> e16; std::vector<CsrEntry> e32;
+                for (int j = 0; j < H; ++j)
+                    for (int q = 0; q < 4; ++q) {
+                        const int r = q * H + j;
+                        int cnt = 0;
+                        for (int e = ch.rowptr[r]; e < ch.rowptr[r + 1]; ++e, ++cnt) {
+                            if (bf16) e16.push_back(((unsigned)ch.col[e] << 16) | f32_to_bf16_rne(ch.val[e]));
+                            else e32.push_back(CsrEntry{ch.val[e], ch.col[e]});
+                        }
+                        for (; cnt % 4; ++cnt) { if (bf16) e16.push_back(0u); else e32.push_back(CsrEntry{0.0f, 0}); }
+                        ptr[(size_t)j * 4 + q + 1] = (int)(bf16 ? e16.size() : e32.size());
+                    }
+                for (int c = 0; c < h->ncta_dir; ++c) {
+                    int u0, n; unit_range_host(H, h->ncta_dir, c, u0, n);
+                    ly.csr_max_slice_entries = std::max(ly.csr_max_slice_entries, ptr[4 * (u0 + n)] - ptr[4 * u0]);
+                }
+                rc = upload(h, &ly.wh_ptr[d], ptr.data(), ptr.size() * sizeof(int), st, "recurrent CSR offsets");
+                if (rc == LSTM_OK) {
+                    if (bf16) rc = upload(h, (unsigned **)&ly.wh_ent[d], e16.data(), e16.size() * 4, st, "recurrent CSR entries");
+                    else rc = upload(h, (CsrEntry **)&ly.wh_ent[d], e32.data(), e32.size() * 8, st, "recurrent CSR entries");
+                }
+                if (rc == LSTM_OK) cudaStreamSynchronize(st);
+            }
+        }
+        if (rc) break;
+        rc = upload(h, &ly.bias, bias_p.data(), bias_p.size() * 4, st, "bias");
+        if (rc == LSTM_OK && !csr)
+            rc = bf16 ? upload(h, (uint16_t **)&ly.wx, wx16.data(), wx16.size() * 2, st, "input weights")
+                      : upload(h, (float **)&ly.wx, wx32.data(), wx32.size() * 4, st, "input weights");
+        if (rc == LSTM_OK && csr) {
+            rc = upload(h, &ly.wx_rowptr, px_rowptr.data(), px_rowptr.size() * sizeof(int), st, "input CSR offsets");
+            if (rc == LSTM_OK) rc = upload(h, &ly.wx_ent, px_ent.data(), px_ent.size() * sizeof(CsrEntry), st, "input CSR entries");
+        }
+        if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)
+            rc = fail(h, LSTM_ERR_CUDA, "upload failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+    if (rc) return bail(rc);
+
+    // workspace
+    const size_t Mmax = (size_t)max_T * max_B;
+    const size_t N = (size_t)D * 4 * H;
+    h->G_cap = std::max(Mmax * N, std::min<size_t>(Mmax, 256) * N * n_split_cap());
+    rc = dev_alloc(h, &h->G, h->G_cap * 4, false, st, "projection workspace");
+    if (rc == LSTM_OK && h->use_tc) {
+        h->ld0 = round_up(in_dim, 8);
+        rc = dev_alloc(h, &h->xb0, Mmax * h->ld0 * 2, true, st, "bf16 input staging");
+        if (rc == LSTM_OK && layers > 1) {
+            h->ldn = round_up(D * H, 8);
+            for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->xbn[i], Mmax * h->ldn * 2, true, st, "bf16 layer activations");
+        }
+    }
+    if (rc == LSTM_OK && layers > 1)
+        for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->ybuf[i], Mmax * D * H * 4, false, st, "layer activations");
+    h->xch_words = (size_t)D * 2 * max_B * H;
+    if (rc == LSTM_OK) rc = dev_alloc(h, &h->xch, h->xch_words * 8, true, st, "exchange buffer");
+    if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
+    if (rc == LSTM_OK) {
+        cudaError_t e = csr ? recur_csr_prepare(h->smem_optin - 64) : recur_dense_prepare(h->smem_optin - 64);
+        if (e == cudaSuccess && h->use_tc) e = proj_tc_prepare();
+        if (e != cudaSuccess) rc = fail(h, LSTM_ERR_CUDA, "kernel set-up failed: %s", cudaGetErrorString(e));
+    }
+    if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)
+        rc = fail(h, LSTM_ERR_CUDA, "workspace set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
+    if (rc) return bail(rc);
+    *out = h;
+    return LSTM_OK;
+}
+
+static int record(lstm_handle *h, int kind, cudaStream_t st)
+{
+    if (!h->prof) return 0;
+    if (h->ev_used >= (int)h->ev.size()) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return 1;
+        h->ev.push_back(e);
+        h->ev_kind.push_back(kind);
+    }
+    h->ev_kind[h->ev_used] = kind;
+    return cudaEventRecord(h->ev[h->ev_used++], st) != cudaSuccess;
+}
+
+int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, const float *c0,
+                 float *y, float *hT, float *cT, void *cuda_stream)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    if (T < 0 || B < 0 || T > h->max_T || B > h->max_B)
+        return fail(h, LSTM_ERR_INVALID, "T=%d B=%d outside [0,%d] x [0,%d]", T, B, h->max_T, h->max_B);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    h->last_stream = st;
+    const int L = h->L, D = h->D, H = h->H;
+    const size_t state_n = (size_t)L * D * B * H;
+    h->ev_used = 0;
+    h->last_launches = 0;
+    if (T == 0 || B == 0) {
+        if (B > 0 && state_n) {
+            for (int i = 0; i < 2; ++i) {
+                float *dst = i ? cT : hT;
+                const float *src = i ? c0 : h0;
+                if (!dst) continue;
+                cudaError_t e = src ? cudaMemcpyAsync(dst, src, state_n * 4, cudaMemcpyDeviceToDevice, st)
+                                    : cudaMemsetAsync(dst, 0, state_n * 4, st);
+                if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "state copy failed: %s", cudaGetErrorString(e));
+            }
+        }
+        return LSTM_OK;
+    }
+    if (!x || !y) return fail(h, LSTM_ERR_INVALID, "x and y must not be NULL");
+
+    const int M = T * B;
+    const bool bf16 = h->dtype == LSTM_BF16W_F32S;
+    const bool csr = h->exec_mode == LSTM_CSR;
+    cudaError_t e = cudaSuccess;
+
+    // stamps of the exchange words must stay unique: restart from a cleared buffer before wrapping
+    if ((unsigned long long)h->stamp_next + (unsigned long long)L * T + 2ull >= 0xffffffffull) {
+        if (cudaMemsetAsync(h->xch, 0, h->xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
+        h->stamp_next = 0;
+    }
+
+    for (int l = 0; l < L; ++l) {
+        Layer &ly = h->layers[l];
+        const float *Xf = l == 0 ? x : h->ybuf[(l - 1) & 1];
+        const int N = D * 4 * H;
+        int nsplit = 1;
+        // ---- input staging + projection
+        if (csr) {
+            if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_proj_csr(Xf, ly.wx_rowptr, ly.wx_ent, ly.bias, h->G, M, N, ly.in_l, !bf16, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        } else if (h->use_tc) {
+            __nv_bfloat16 *xb = l == 0 ? h->xb0 : h->xbn[(l - 1) & 1];
+            if (l == 0) {
+                if (record(h, LSTM_K_STAGE, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+                e = launch_stage_bf16(x, xb, M, h->in_dim, h->ld0, st);
+                ++h->last_launches;
+                if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+                if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "staging launch failed: %s", cudaGetErrorString(e));
+            }
+            if (ly.plan_M != M) {
+                char msg[256];
+                if (proj_tc_plan(&ly.plan, (const __nv_bfloat16 *)ly.wx, xb, M, N, ly.in_l, ly.ldk, h->sm_count, msg, sizeof msg))
+                    return fail(h, LSTM_ERR_CUDA, "tensor-core projection plan failed: %s", msg);
+                ly.plan_M = M;
+            }
+            nsplit = ly.plan.nsplit;
+            if ((size_t)nsplit * M * N > h->G_cap) return fail(h, LSTM_ERR_CUDA, "internal: projection workspace too small");
+            if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_proj_tc(ly.plan, ly.bias, h->G, h->status_dev, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        } else {
+            if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_proj_simt(Xf, ly.wx, bf16, ly.ldk, ly.bias, h->G, M, N, ly.in_l, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        }
+        if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "projection launch failed (layer %d): %s", l, cudaGetErrorString(e));
+
+        // ---- recurrence
+        const RecurShape shp = recur_shape(h, B, l);
+        RecurArgs a;
+        memset(&a, 0, sizeof a);
+        a.H = H; a.Hp8 = h->Hp8; a.Hs = h->Hs; a.B = B; a.T = T; a.D = D;
+        a.ncta_dir = h->ncta_dir; a.nsplit = nsplit; a.BT = shp.BT; a.w_smem_bytes = shp.w_smem_bytes;
+        a.stamp_base = h->stamp_next;
+        h->stamp_next += (unsigned)T + 1u;
+        a.spin_limit = h->spin_limit;
+        for (int d = 0; d < D; ++d) { a.wh[d] = ly.wh[d]; a.csr_ptr[d] = ly.wh_ptr[d]; a.csr_ent[d] = ly.wh_ent[d]; }
+        a.G = h->G;
+        a.g_split_stride = (long long)M * N;
+        const size_t soff = (size_t)l * D * B * H;
+        a.h0 = h0 ? h0 + soff : nullptr; a.c0 = c0 ? c0 + soff : nullptr;
+        a.hT = hT ? hT + soff : nullptr; a.cT = cT ? cT + soff : nullptr;
+        a.y = l == L - 1 ? y : h->ybuf[l & 1];
+        a.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
+        a.xb_ld = h->ldn;
+        a.xch = h->xch;
+        a.status = h->status_dev;
+        if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        e = csr ? launch_recur_csr(a, bf16, h->threads, shp.smem, st) : launch_recur_dense(a, bf16, h->threads, shp.smem, st);
+        ++h->last_launches;
+        if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
+    }
+    return LSTM_OK;
+}
+
+int lstm_status(lstm_handle *h)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    int v = 0;
+    cudaError_t e = cudaStreamSynchronize(h->last_stream);
+    if (e == cudaSuccess) e = cudaMemcpy(&v, h->status_dev, sizeof v, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "status read failed: %s", cudaGetErrorString(e));
+    if (v != 0) {
+        cudaMemset(h->status_dev, 0, sizeof v);
+        return fail(h, v, v == LSTM_ERR_TIMEOUT ? "a device-side wait gave up (timeout); outputs are undefined" : "device reported status %d", v);
+    }
+    return LSTM_OK;
+}
+
+int lstm_forward_host(lstm_handle *h, const float *x, int T, int B, const float *h0, const float *c0,
+                      float *y, float *hT, float *cT, void *cuda_stream)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    if (T < 0 || B < 0 || T > h->max_T || B > h->max_B)
+        return fail(h, LSTM_ERR_INVALID, "T=%d B=%d outside [0,%d] x [0,%d]", T, B, h->max_T, h->max_B);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t Mmax = (size_t)h->max_T * h->max_B;
+    const size_t smax = (size_t)h->L * h->D * h->max_B * h->H;
+    if (!h->hx) {
+        int rc = dev_alloc(h, &h->hx, Mmax * h->in_dim * 4, false, st, "host-variant x");
+        if (!rc) rc = dev_alloc(h, &h->hy, Mmax * h->D * h->H * 4, false, st, "host-variant y");
+        if (!rc) rc = dev_alloc(h, &h->hh0, smax * 4, false, st, "host-variant h0");
+        if (!rc) rc = dev_alloc(h, &h->hc0, smax * 4, false, st, "host-variant c0");
+        if (!rc) rc = dev_alloc(h, &h->hhT, smax * 4, false, st, "host-variant hT");
+        if (!rc) rc = dev_alloc(h, &h->hcT, smax * 4, false, st, "host-variant cT");
+        if (rc) return rc;
+    }
+    const size_t xn = (size_t)T * B * h->in_dim, yn = (size_t)T * B * h->D * h->H, sn = (size_t)h->L * h->D * B * h->H;
+    cudaError_t e = cudaSuccess;
+    if (xn && !x) return fail(h, LSTM_ERR_INVALID, "x must not be NULL");
+    if (yn && !y) return fail(h, LSTM_ERR_INVALID, "y must not be NULL");
+    if (xn) e = cudaMemcpyAsync(h->hx, x, xn * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && h0 && sn) e = cudaMemcpyAsync(h->hh0, h0, sn * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && c0 && sn) e = cudaMemcpyAsync(h->hc0, c0, sn * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(e));
+    int rc = lstm_forward(h, h->hx, T, B, h0 ? h->hh0 : nullptr, c0 ? h->hc0 : nullptr, h->hy,
+                          hT ? h->hhT : nullptr, cT ? h->hcT : nullptr, cuda_stream);
+    if (rc) return rc;
+    if (yn) e = cudaMemcpyAsync(y, h->hy, yn * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && hT && sn) e = cudaMemcpyAsync(hT, h->hhT, sn * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && cT && sn) e = cudaMemcpyAsync(cT, h->hcT, sn * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(e));
+    return lstm_status(h);
+}
+
+int lstm_destroy(lstm_handle *h)
+{
+    if (!h) return LSTM_OK;
+    cudaDeviceSynchronize();
+    free_all(h);
+    delete h;
+    return LSTM_OK;
+}
+
+int lstm_profile_enable(lstm_handle *h, int on)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    h->prof = on != 0;
+    h->ev_used = 0;
+    return LSTM_OK;
+}
+
+int lstm_profile_read(lstm_handle *h, int *launches, float *ms)
+{
+    if (!h || !launches || !ms) return LSTM_ERR_INVALID;
+    for (int k = 0; k < LSTM_K_COUNT; ++k) { launches[k] = 0; ms[k] = 0.0f; }
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess)
+        return fail(h, LSTM_ERR_CUDA, "synchronise failed: %s", cudaGetErrorString(cudaGetLastError()));
+    for (int i = 0; i + 1 < h->ev_used; i += 2) {
+        const int k = h->ev_kind[i];
+        float t = 0.0f;
+        if (k < 0 || k >= LSTM_K_COUNT) continue;
+        if (cudaEventElapsedTime(&t, h->ev[i], h->ev[i + 1]) != cudaSuccess)
+            return fail(h, LSTM_ERR_CUDA, "event timing failed: %s", cudaGetErrorString(cudaGetLastError()));
+        launches[k] += 1;
+        ms[k] += t;
+    }
+    return LSTM_OK;
+}
+
+int lstm_info(const lstm_handle *h, int64_t *out, int n)
+{
+    if (!h || !out || n < 0) return 0;
+    const RecurShape shp = recur_shape(h, h->max_B, 0);
+    const size_t wsize = h->dtype == LSTM_BF16W_F32S ? 2 : 4;
+    int64_t rows_res = 0, rows_str = 0;
+    if (h->exec_mode == LSTM_DENSE) {
+        const size_t unit_bytes = (size_t)4 * h->Hp8 * wsize;
+        const int ures = (int)std::min<size_t>(h->upc, shp.w_smem_bytes / unit_bytes);
+        rows_res = 4 * ures; rows_str = 4 * (h->upc - ures);
+    }
+    const Layer &l0 = h->layers[0];
+    const int launches = h->L * 2 + (h->use_tc ? 1 : 0);
+    const int64_t vals[9] = {h->sm_count, h->ncta_dir, h->threads, (int64_t)shp.smem, rows_res, rows_str,
+                             (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches};
+    for (int i = 0; i < n && i < 9; ++i) out[i] = vals[i];
+    return 9;
+}
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// Shared declarations of the lstm_b200 library: kernel argument blocks and launch entry points.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace lstm {
+
+// device status word values (mirrors the LSTM_* return codes of the C header)
+constexpr int kStatusOk = 0;
+constexpr int kStatusTimeout = 5;
+
+// ---------------------------------------------------------------------------------------------------
+// Recurrent kernel (dense and CSR).  One cooperative launch per layer covers both directions: CTAs
+// [0, ncta_dir) run direction 0, CTAs [ncta_dir, 2*ncta_dir) direction 1.  Hidden units are split
+// evenly over a direction's CTAs; CTA c owns units [u0(c), u0(c) + n(c)).
+// ---------------------------------------------------------------------------------------------------
+struct RecurArgs {
+    int H;              // hidden width
+    int Hp8;            // dense: row length of the packed recurrent matrix (H rounded up to 8)
+    int Hs;             // length of one staged h row in shared memory (H rounded up to 256)
+    int B, T, D;
+    int ncta_dir;       // CTAs per direction
+    int nsplit;         // partial planes of the projection output to add up
+    int BT;             // batch rows processed per chunk (1, 2, 4 or 8)
+    int w_smem_bytes;   // shared-memory bytes set aside for resident weights
+    unsigned stamp_base;        // exchange words of step s carry stamp_base + s + 1
+    long long spin_limit;       // clock64 ticks a wait may last before the kernel gives up
+    // dense: [H][4][Hp8] (unit-major, gates i,f,g,o); element type = weight type
+    const void *wh[2];
+    // CSR: per direction, rows in the same unit-major order; entry_ptr[4H+1] counts entries padded
+    // per row to a multiple of 4; entries are {col<<16 | bf16} words (bf16) or {val, col} pairs (fp32)
+    const int *csr_ptr[2];
+    const void *csr_ent[2];
+    const float *G;             // [nsplit][T*B][D][H][4] projection output incl. bias
+    long long g_split_stride;   // elements between partial planes
+    const float *h0, *c0;       // [D][B][H] of this layer or nullptr
+    float *hT, *cT;             // [D][B][H] of this layer or nullptr
+    float *y;                   // [T][B][D*H]
+    __nv_bfloat16 *xb_next;     // bf16 copy of y for the next layer's projection, or nullptr
+    int xb_ld;                  // its row stride in elements
+    unsigned long long *xch;    // [D][2][B][H] exchange words {stamp:32 | h bits:32}
+    int *status;                // device status word
+};
+
+cudaError_t launch_recur_dense(const RecurArgs &a, bool bf16_weights, int threads, size_t smem,
+                               cudaStream_t st);
+cudaError_t launch_recur_csr(const RecurArgs &a, bool bf16_weights, int threads, size_t smem,
+                             cudaStream_t st);
+cudaError_t recur_dense_prepare(int max_smem);   // raises the dynamic shared-memory limit once
+cudaError_t recur_csr_prepare(int max_smem);
+
+// ---------------------------------------------------------------------------------------------------
+// Input staging and projection
+// ---------------------------------------------------------------------------------------------------
+// x fp32 [M][K] -> xb bf16 [M][ld] (columns K..ld-1 are written as zero)
+cudaError_t launch_stage_bf16(const float *x, __nv_bfloat16 *xb, long long M, int K, int ld,
+                              cudaStream_t st);
+
+// G[m][n] = sum_k X[m][k] * W[n][k] + bias[n];  X fp32 [M][K], W [N][ldw] fp32 or bf16, G fp32 [M][N]
+cudaError_t launch_proj_simt(const float *X, const void *W, bool bf16_weights, int ldw,
+                             const float *bias, float *G, int M, int N, int K, cudaStream_t st);
+
+// G[m][n] = sum_e val[e] * X[m][col[e]] + bias[n] over CSR row n (entries {val,col} pairs)
+struct CsrEntry { float val; int col; };
+cudaError_t launch_proj_csr(const float *X, const int *rowptr, const CsrEntry *ent,
+                            const float *bias, float *G, int M, int N, int K, bool f64_acc, cudaStream_t st);
+
+// Tensor-core projection (tcgen05 + TMEM + TMA).  A = packed weights [N][ldk] bf16 (K-major),
+// Bm = activations [M][ldk] bf16; writes G[split][M][N] fp32 (+bias on split 0).
+struct ProjTcPlan {
+    alignas(64) unsigned char tmap_w[128];
+    alignas(64) unsigned char tmap_x[128];
+    int M, N, K, ldk;
+    int n_tile;        // MMA N extent (activation rows per tile), multiple of 16, <= 256
+    int nsplit;        // split-K factor
+    int kblocks;       // ceil(K / 64)
+};
+int  proj_tc_plan(ProjTcPlan *p, const __nv_bfloat16 *W, const __nv_bfloat16 *X, int M, int N, int K,
+                  int ldk, int sm_count, char *err, int errlen);
+cudaError_t launch_proj_tc(const ProjTcPlan &p, const float *bias, float *G, int *status,
+                           cudaStream_t st);
+cudaError_t proj_tc_prepare();
+
+}  // namespace lstm

@@ -1,0 +1,50 @@
+"""Helpers shared by the GPU parity tests: run the CUDA library through its C ABI and compare with
+the fp64 oracle on the same seeded inputs."""
+import numpy as np
+
+import lstm_workloads as wl
+
+
+def csr_weights(oracle, weights):
+    """Per (layer, direction): CSR triplets of the kept entries (mask positions, or non-zeros)."""
+    out = []
+    for w in weights:
+        out.append({"wx_csr": oracle.dense_to_csr(w["wx"], w.get("mask_x")),
+                    "wh_csr": oracle.dense_to_csr(w["wh"], w.get("mask_h")), "b": w.get("b")})
+    return out
+
+
+def run_gpu(w: wl.Workload, weights, x, h0=None, c0=None, exec_mode="dense", max_T=None, max_B=None,
+            chunks=None):
+    """Returns (y, hT, cT) as numpy arrays.  ``chunks``: split T into consecutive calls carrying state."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    m = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
+                 exec_mode=exec_mode, max_T=max_T or max(w.T, 1), max_B=max_B or max(w.B, 1))
+    try:
+        dev = torch.device("cuda:0")
+        xt = torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(dev)
+        h = torch.from_numpy(np.ascontiguousarray(h0, np.float32)).to(dev) if h0 is not None else None
+        c = torch.from_numpy(np.ascontiguousarray(c0, np.float32)).to(dev) if c0 is not None else None
+        if chunks is None:
+            y, hT, cT = m.forward(xt, h, c)
+            m.check()
+        else:
+            ys, t0 = [], 0
+            for n in chunks:
+                yy, h, c = m.forward(xt[t0:t0 + n].contiguous(), h, c)
+                m.check()
+                ys.append(yy)
+                t0 += n
+            y, hT, cT = torch.cat(ys), h, c
+        torch.cuda.synchronize()
+        return y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()
+    finally:
+        m.close()
+
+
+def assert_close(got, ref, dtype, what=""):
+    tol = wl.TOLERANCE[dtype]
+    for name, g, r in zip(("y", "hT", "cT"), got, ref):
+        floored, scaled = wl.rel_err(g, r)
+        assert floored <= tol, f"{what} {name}: floored rel err {floored:.3e} (scaled {scaled:.3e}) > {tol}"

@@ -1,0 +1,182 @@
+"""CUDA library vs fp64 oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+
+import lstm_workloads as wl
+from gpu_util import assert_close, csr_weights, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, L, bidir, in_dim, H, T, B, dtype, density=1.0, seed=1):
+    return wl.Workload(name, L, bidir, in_dim, H, T, B, dtype, 0.3, density=density, seed=seed)
+
+
+# awkward shapes: H not a multiple of 8/32/148, H = 1, T = 1, B not a power of two, in != H
+SHAPES = [
+    small("h1", 1, False, 1, 1, 3, 1, "fp32"),
+    small("h2_bidir", 2, True, 3, 2, 3, 2, "fp32"),
+    small("h7_b3", 2, False, 5, 7, 4, 3, "fp32"),
+    small("t1", 1, True, 9, 33, 1, 5, "bf16"),
+    small("h100_b1", 1, False, 40, 100, 6, 1, "bf16"),
+    small("h149_b2", 2, False, 64, 149, 5, 2, "bf16"),
+    small("h300_b5", 1, True, 77, 300, 7, 5, "bf16"),
+    small("h300_b16", 1, False, 96, 300, 5, 16, "fp32"),
+    small("h200_b20", 3, True, 50, 200, 4, 20, "bf16"),
+    small("h513_b9", 1, False, 130, 513, 3, 9, "bf16"),
+]
+
+
+@pytest.mark.parametrize("w", SHAPES, ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", ["dense", "csr"])
+def test_small_shapes(oracle, w, mode):
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got = run_gpu(w, weights, x, h0, c0, exec_mode=mode)
+    assert_close(got, ref, w.dtype, f"{w.name}/{mode}")
+
+
+@pytest.mark.parametrize("mode", ["dense", "csr"])
+def test_masked_small(oracle, mode):
+    w = small("masked", 2, True, 60, 90, 6, 3, "bf16", density=0.2, seed=5)
+    weights, x = wl.make(w)
+    weights[0]["mask_h"][5] = 0                      # an empty recurrent row
+    weights[0]["wh"][5] = 0
+    ref = oracle.forward(weights, x, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got = run_gpu(w, weights if mode == "dense" else csr_weights(oracle, weights), x, exec_mode=mode)
+    assert_close(got, ref, w.dtype, mode)
+
+
+def test_masks_apply_as_zeros_in_dense_mode(oracle):
+    """A mask handed to the dense path multiplies the weights (W (x) Msk), it is not ignored."""
+    w = small("maskapply", 1, False, 20, 24, 5, 2, "fp32", seed=6)
+    weights, x = wl.make(w)
+    rng = np.random.default_rng(1)
+    mx = (rng.random(weights[0]["wx"].shape) < 0.5).astype(np.uint8)
+    mh = (rng.random(weights[0]["wh"].shape) < 0.5).astype(np.uint8)
+    masked = [{**weights[0], "mask_x": mx, "mask_h": mh}]
+    ref = oracle.forward(masked, x, layers=1, bidir=False, hidden=w.hidden)
+    for mode in ("dense", "csr"):
+        assert_close(run_gpu(w, masked, x, exec_mode=mode), ref, "fp32", mode)
+
+
+def test_chunked_calls_carry_state(oracle):
+    w = small("chunk", 2, False, 30, 70, 12, 3, "bf16", seed=7)
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=2, bidir=False, hidden=w.hidden)
+    got = run_gpu(w, weights, x, chunks=[5, 1, 6])
+    assert_close(got, ref, "bf16", "chunked")
+    wb = w.with_(bidir=True, layers=1)
+    weights, x = wl.make(wb)
+    h0, c0 = wl.make_states(wb)
+    ref = oracle.forward(weights, x, h0, c0, layers=1, bidir=True, hidden=w.hidden)
+    assert_close(run_gpu(wb, weights, x, h0, c0, max_T=20, max_B=6), ref, "bf16", "larger workspace")
+
+
+def test_empty_sequence_and_batch(oracle):
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = small("empty", 1, False, 4, 6, 3, 2, "fp32")
+    weights, x = wl.make(w)
+    m = pkg.LSTM(weights, layers=1, in_dim=4, hidden=6, dtype="fp32", max_T=4, max_B=2)
+    h0, c0 = wl.make_states(w)
+    h = torch.from_numpy(h0).cuda(); c = torch.from_numpy(c0).cuda()
+    y, hT, cT = m.forward(torch.empty((0, 2, 4), device="cuda"), h, c)
+    m.check()
+    assert y.shape == (0, 2, 6) and torch.equal(hT, h) and torch.equal(cT, c)
+    y, hT, cT = m.forward(torch.empty((3, 0, 4), device="cuda"))
+    m.check()
+    assert y.shape == (3, 0, 6)
+    with pytest.raises(pkg.LstmError):
+        m.forward(torch.zeros((5, 2, 4), device="cuda"))          # T > max_T
+    with pytest.raises(pkg.LstmError):
+        m.forward(torch.zeros((1, 3, 4), device="cuda"))          # B > max_B
+    m.close()
+
+
+def test_bad_csr_is_rejected():
+    import paper_1901_10997_b200 as pkg
+    H, in_dim = 3, 2
+    rp = np.array([0, 2] + [2] * (4 * H - 1), np.int32)
+    bad = {"wx_csr": (rp, np.array([1, 0], np.int32), np.ones(2, np.float32)),     # unsorted columns
+           "wh": np.zeros((4 * H, H), np.float32)}
+    with pytest.raises(pkg.LstmError) as e:
+        pkg.LSTM([bad], layers=1, in_dim=in_dim, hidden=H, dtype="fp32", exec_mode="csr", max_T=2, max_B=1)
+    assert e.value.code == pkg.LSTM_ERR_INVALID
+    bad["wx_csr"] = (rp, np.array([0, 7], np.int32), np.ones(2, np.float32))          # out of range
+    with pytest.raises(pkg.LstmError):
+        pkg.LSTM([bad], layers=1, in_dim=in_dim, hidden=H, dtype="fp32", exec_mode="csr", max_T=2, max_B=1)
+
+
+def test_host_buffer_call_matches_device_call(oracle):
+    import paper_1901_10997_b200 as pkg
+    w = small("host", 2, False, 33, 65, 6, 4, "bf16", seed=9)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=2, bidir=False, hidden=w.hidden)
+    m = pkg.LSTM(weights, layers=2, in_dim=w.in_dim, hidden=w.hidden, dtype="bf16", max_T=w.T, max_B=w.B)
+    got = m.forward_host(x, h0, c0)
+    assert_close(got, ref, "bf16", "host")
+    m.close()
+
+
+# ---------------------------------------------------------------- the five configurations
+def test_config1_full(oracle):
+    w = wl.config1()
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    assert_close(run_gpu(w, weights, x), ref, w.dtype, w.name)
+
+
+def test_config2_b1_full(oracle):
+    w = wl.config2(1)
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    assert_close(run_gpu(w, weights, x), ref, w.dtype, w.name)
+
+
+def test_config2_b20_sampled_columns(oracle):
+    """Full size on the GPU; batch columns are independent, so the oracle checks three of them."""
+    w = wl.config2(20)
+    weights, x = wl.make(w)
+    y, hT, cT = run_gpu(w, weights, x)
+    for b in (0, 7, 19):
+        ref = oracle.forward(weights, x[:, b:b + 1], layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        assert_close((y[:, b:b + 1], hT[:, b:b + 1], cT[:, b:b + 1]), ref, w.dtype, f"{w.name} col {b}")
+
+
+@pytest.mark.parametrize("H", [128, 136, 600, 1184, 1192, 1896, 2048])
+def test_config3_points(oracle, H):
+    w = wl.config3(H)
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=1, bidir=False, hidden=H)
+    assert_close(run_gpu(w, weights, x), ref, w.dtype, w.name)
+
+
+@pytest.mark.parametrize("density", [0.10, 0.05])
+def test_config4_dense_with_zeros_vs_csr(oracle, density):
+    w = wl.config4(density)
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    dense = run_gpu(w, weights, x, exec_mode="dense")
+    sparse = run_gpu(w, weights, x, exec_mode="csr")
+    assert_close(dense, ref, w.dtype, "dense-with-zeros")
+    assert_close(sparse, ref, w.dtype, "csr")
+    assert_close(sparse, dense, w.dtype, "csr vs dense")
+
+
+def test_config5_b1_full(oracle):
+    w = wl.config5(1)
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    assert_close(run_gpu(w, weights, x), ref, w.dtype, w.name)
+
+
+def test_config5_b16_sampled_columns(oracle):
+    w = wl.config5(16)
+    weights, x = wl.make(w)
+    y, hT, cT = run_gpu(w, weights, x)
+    for b in (3, 15):
+        ref = oracle.forward(weights, x[:, b:b + 1], layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        assert_close((y[:, b:b + 1], hT[:, b:b + 1], cT[:, b:b + 1]), ref, w.dtype, f"{w.name} col {b}")
