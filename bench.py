@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the stacked-LSTM forward pass on B200.
+
+Default run (one JSON line on stdout):
+    python bench.py [--gpus N] [--steps K] [--warmup W]
+A step is one lstm_forward over the large language-model workload (2 layers, 1500 -> 1500, T = 35,
+batch 1, bf16 weights / fp32 state): input projection for all timesteps + serial recurrence, every
+layer.  `value` is microseconds per sequence with inputs resident in device memory; `e2e` is the same
+through lstm_forward_host with pinned host buffers (copies inside the timed region).  With N > 1 each
+rank runs an independent replica (batch columns and sequences never interact): no collective on the
+data path, N sequences per step.
+
+Other modes:
+    --impl reference     time the fp64 CPU oracle on the same workload (host cores only)
+    --sweep              latency vs hidden size (H = 128..2048 step 8) with the LHP analysis
+    --workload NAME      cfg1 | cfg2 | cfg2_b20 | cfg4_10 | cfg4_05 | cfg4_10_csr | cfg4_05_csr |
+                         cfg5 | cfg5_b16 (default cfg2)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import lstm_workloads as wl  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+
+
+def pick_workload(name: str):
+    table = {
+        "cfg1": (wl.config1(), "dense"),
+        "cfg2": (wl.config2(1), "dense"),
+        "cfg2_b20": (wl.config2(20), "dense"),
+        "cfg4_10": (wl.config4(0.10), "dense"),
+        "cfg4_05": (wl.config4(0.05), "dense"),
+        "cfg4_10_csr": (wl.config4(0.10), "csr"),
+        "cfg4_05_csr": (wl.config4(0.05), "csr"),
+        "cfg5": (wl.config5(1), "dense"),
+        "cfg5_b16": (wl.config5(16), "dense"),
+    }
+    return table[name]
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            d = json.loads(p.read_text())
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def recurrence_bytes_per_launch(w: wl.Workload, nnz_per_layer=None) -> float:
+    """Algorithmic bytes one recurrent-kernel launch (one layer, all T steps, all directions) needs if
+    nothing were resident: per step and direction the recurrent matrix once (4H*H*w bytes dense, or
+    nnz*(value + 16-bit column) + row offsets for CSR), h read and written (B*H*8), and the
+    projection row read (B*4H*4)."""
+    H, B, T, D = w.hidden, w.B, w.T, w.dirs
+    wbytes = 2 if w.dtype == "bf16" else 4
+    if nnz_per_layer is None:
+        mat = 4.0 * H * H * wbytes
+    else:
+        mat = nnz_per_layer / D * (wbytes + 2) + (4 * H + 1) * 4
+    return T * D * (mat + B * H * 8.0 + B * 4.0 * H * 4.0)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if r & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.01)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_time(w: wl.Workload, weights, x, target_seconds=12.0, max_reps=50):
+    """Times the oracle as it stands on a bounded sample: whole sequences of the workload (for B > 1
+    only the first batch column), repeated until ~target_seconds of wall time have passed."""
+    import oracle
+    xs = x[:, :1] if w.B > 1 else x
+    t0 = time.perf_counter()
+    oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    first = time.perf_counter() - t0
+    reps = int(max(1, min(max_reps, target_seconds / max(first, 1e-6))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    per_seq = (time.perf_counter() - t0) / reps
+    return per_seq, reps, oracle.threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w, _mode = pick_workload(args.workload)
+    weights, x = wl.make(w)
+    import oracle
+    xs = x[:, :1] if w.B > 1 else x
+    for _ in range(min(args.warmup, 1)):
+        oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    steps = max(1, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    per_seq = (time.perf_counter() - t0) / steps
+    us = per_seq * 1e6
+    sample = f"{steps} whole sequences of {w.name} (T={w.T}, one batch column per step), fp64 oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": "us_per_sequence", "value": us, "unit": "us", "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": per_seq * 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.layers, "hidden": w.hidden, "T": w.T, "B": 1},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def flush_l2(buf):
+    buf.zero_()
+
+
+def time_steps(fn, steps, warmup, flush_buf, torch):
+    """Per-step CUDA-event timing on the current stream; L2 is flushed between steps outside the
+    event pairs.  Returns the list of per-step milliseconds."""
+    for _ in range(warmup):
+        flush_l2(flush_buf)
+        fn()
+    torch.cuda.synchronize()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for i in range(steps):
+        flush_l2(flush_buf)
+        starts[i].record()
+        fn()
+        ends[i].record()
+    torch.cuda.synchronize()
+    return [s.elapsed_time(e) for s, e in zip(starts, ends)]
+
+
+def run_gpu(args):
+    import torch
+    import paper_1901_10997_b200 as pkg
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    w, mode = pick_workload(args.workload)
+    weights, x = wl.make(w)
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        per_seq, reps, cores = oracle_time(w, weights, x)
+        cpu = {"value": per_seq * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+               "sample": f"{reps} whole sequences of {w.name} (T={w.T}, one batch column each) after one warm-up"}
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+
+    model = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
+                     exec_mode=mode, max_T=w.T, max_B=w.B)
+    dev = torch.device("cuda", local_rank)
+    xd = torch.from_numpy(x).to(dev)
+    out = (torch.empty((w.T, w.B, w.dirs * w.hidden), device=dev),
+           torch.empty((w.layers * w.dirs, w.B, w.hidden), device=dev),
+           torch.empty((w.layers * w.dirs, w.B, w.hidden), device=dev))
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def step():
+        model.forward(xd, out=out)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- timed region: device-resident inputs
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        ms = time_steps(step, args.steps, max(args.warmup, 3), flush_buf, torch)
+    barrier()
+    model.check()
+    total_ms = sum(ms)
+    launches_per_fwd = model.info()["launches_per_forward"]
+
+    # ---- same region again with the library's per-kernel events, for the roofline of the dominant kernel
+    model.profile_enable(True)
+    rec_ms, rec_n, proj_ms, stage_ms = 0.0, 0, 0.0, 0.0
+    for i in range(args.steps + 3):
+        flush_l2(flush_buf)
+        step()
+        n, t = model.profile_read()
+        if i >= 3:
+            rec_ms += t[pkg.LSTM_K_RECUR]; rec_n += n[pkg.LSTM_K_RECUR]
+            proj_ms += t[pkg.LSTM_K_PROJ]; stage_ms += t[pkg.LSTM_K_STAGE]
+    model.profile_enable(False)
+
+    # ---- end to end through the host-buffer entry point (pinned buffers, copies inside the timing)
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.empty((w.T, w.B, w.dirs * w.hidden)).pin_memory()
+    hTh = torch.empty((w.layers * w.dirs, w.B, w.hidden)).pin_memory()
+    cTh = torch.empty_like(hTh).pin_memory()
+    st = torch.cuda.current_stream().cuda_stream
+    for _ in range(3):
+        model.forward_host(xh, y=yh, hT=hTh, cT=cTh, stream=st)
+    barrier()
+    e2e_steps = args.steps
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        flush_l2(flush_buf)
+        model.forward_host(xh, y=yh, hT=hTh, cT=cTh, stream=st)
+    torch.cuda.synchronize()
+    e2e_total = time.perf_counter() - t0
+    # the flush is outside the metric: time it separately and subtract
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        flush_l2(flush_buf)
+    torch.cuda.synchronize()
+    e2e_total -= time.perf_counter() - t0
+    barrier()
+
+    tot = torch.tensor([total_ms, e2e_total * 1e3], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(tot, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(tot[0]), float(tot[1])
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        seqs = world * w.B
+        us_per_seq = ms_per_step * 1e3 / seqs
+        peak, peak_kind = measured_peaks()
+        nnz = None
+        if mode == "csr":
+            nnz = float(np.mean([sum(int(np.count_nonzero(weights[l * w.dirs + d]["mask_h"])) for d in range(w.dirs))
+                                 for l in range(w.layers)]))
+        alg_bytes = recurrence_bytes_per_launch(w, nnz)
+        rec_avg_ms = rec_ms / max(rec_n, 1)
+        achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
+        traffic = None
+        tp = ROOT / "profiles" / "traffic.json"
+        if tp.exists():
+            try:
+                traffic = json.loads(tp.read_text()).get(f"recur/{args.workload}")
+            except Exception:
+                traffic = None
+        line = {
+            "metric": "us_per_sequence", "value": us_per_seq, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.layers, "dirs": w.dirs, "in_dim": w.in_dim, "hidden": w.hidden,
+                       "T": w.T, "B": w.B, "exec_mode": mode, "weights": w.dtype, "state": "fp32", "l2": "flushed between timed steps (256 MiB write)",
+                       "parallelism": f"replicas x{world}"},
+            "sequences_per_sec": seqs / (ms_per_step * 1e-3),
+            "step_ms_p10_p50_p90": [float(np.percentile(ms, q)) for q in (10, 50, 90)],
+            "clocks": clocks.summary(),
+            "gpu_launches": int(launches_per_fwd * args.steps),
+            "e2e": {"value": e2e_ms * 1e3 / e2e_steps / seqs, "unit": "us",
+                    "h2d_bytes_per_step": int(x.nbytes),
+                    "d2h_bytes_per_step": int(yh.numel() * 4 + hTh.numel() * 4 + cTh.numel() * 4)},
+            "roofline": {"bound": "hbm", "kernel": "recur_kernel (one launch = one layer, all T steps)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": (achieved / peak if achieved else None), "peak_kind": f"of {peak_kind}",
+                         "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
+                         "avg_launch_ms": rec_avg_ms,
+                         "us_per_timestep": rec_avg_ms * 1e3 / w.T,
+                         "note": "weights are resident in shared memory, so the fraction of the HBM "
+                                 "weight-read bound may exceed 1"},
+            "kernel_ms_per_forward": {"stage": stage_ms / args.steps, "projection": proj_ms / args.steps,
+                                      "recurrence": rec_ms / args.steps},
+            "library": model.info(),
+        }
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    model.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def lhp_analysis(hs, lat, eps):
+    """Latency-hysteresis points (paper, Section 3): scanning from the largest size down, a size is an
+    LHP if no larger size is at most (1+eps) times as slow; every other size is dominated (a larger
+    model runs at least as fast).  Redundancy = (1 - #LHP / #points) * 100 %."""
+    lhps, best = [], float("inf")
+    for h, t in sorted(zip(hs, lat), reverse=True):
+        if t * (1 + eps) < best:
+            lhps.append(h)
+        best = min(best, t)
+    lhps.sort()
+    return lhps, (1 - len(lhps) / len(hs)) * 100.0
+
+
+def run_sweep(args):
+    import torch
+    import paper_1901_10997_b200 as pkg
+    dev = torch.device("cuda", 0)
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    outdir = ROOT / "gpurun_out"
+    outdir.mkdir(exist_ok=True)
+    sizes = wl.config3_sizes() if not args.sweep_sizes else [int(s) for s in args.sweep_sizes.split(",")]
+    rows = []
+    for H in sizes:
+        w = wl.config3(H)
+        weights, x = wl.make(w)
+        m = pkg.LSTM(weights, layers=1, in_dim=H, hidden=H, dtype="bf16", max_T=w.T, max_B=1)
+        xd = torch.from_numpy(x).to(dev)
+        out = (torch.empty((w.T, 1, H), device=dev), torch.empty((1, 1, H), device=dev), torch.empty((1, 1, H), device=dev))
+        ms = time_steps(lambda: m.forward(xd, out=out), args.steps, max(args.warmup, 3), flush_buf, torch)
+        m.check()
+        err = None
+        if args.sweep_parity:
+            import oracle
+            ref = oracle.forward(weights, x, layers=1, bidir=False, hidden=H)
+            err = max(wl.rel_err(g.cpu().numpy(), r)[0] for g, r in zip(out, ref))
+        info = m.info()
+        m.close()
+        rows.append({"H": H, "us_p50": float(np.percentile(ms, 50)) * 1e3, "us_p10": float(np.percentile(ms, 10)) * 1e3,
+                     "us_p90": float(np.percentile(ms, 90)) * 1e3, "rows_streamed": info["rows_streamed"],
+                     "threads": info["threads"], "max_rel_err": err})
+        print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
+    hs = [r["H"] for r in rows]
+    lat = [r["us_p50"] for r in rows]
+    res = {"workload": "cfg3 sweep: 1 layer, in = hidden = H, T = 35, B = 1, bf16 weights", "steps": args.steps, "points": rows}
+    for eps in (0.0, 0.005):
+        lhps, red = lhp_analysis(hs, lat, eps)
+        res[f"lhp_eps_{eps:g}"] = {"lhps": lhps, "count": len(lhps), "redundancy_percent": red}
+    (outdir / "sweep_cfg3.json").write_text(json.dumps(res, indent=1))
+    print(json.dumps({k: v for k, v in res.items() if k != "points"}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sweep-sizes", default="")
+    ap.add_argument("--sweep-parity", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -106,7 +106,7 @@ LSTM_API int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, 
  *   y  [T,B,D*H]         hT, cT [L*D,B,H] or NULL (not wanted)
  * 0 <= T <= max_T, 0 <= B <= max_B (T = 0 or B = 0: nothing is launched; hT,cT receive h0,c0).
  * Work is enqueued on cuda_stream and the call returns without synchronising; a device-side timeout
- * of this call is reported by the next lstm_forward / lstm_status on the handle.
+ * of this call is reported by lstm_status on the handle.
  * Steps, in order, per layer: input staging (bf16 mode), input projection for all timesteps at once
  * (the x_t half of W [x_t, h_{t-1}] + b), then the serial recurrence with the gate nonlinearities and
  * the c/h update fused into one persistent kernel.
@@ -149,7 +149,7 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
  * [2] threads per CTA, [3] dynamic shared memory bytes per CTA at max_B, [4] recurrent-matrix rows
  * resident in shared memory per CTA (max over CTAs), [5] rows streamed from L2 per CTA (max),
  * [6] split-K factor of the input projection at max_T*max_B, [7] 1 if the projection uses the tensor-core
- * (tcgen05) kernel, [8] kernels launched by one lstm_forward at (max_T, max_B).
+ * (tcgen05) kernel, [8] kernels launched by the most recent lstm_forward (before the first call: the count expected).
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 

@@ -713,7 +713,7 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
         rows_res = 4 * ures; rows_str = 4 * (h->upc - ures);
     }
     const Layer &l0 = h->layers[0];
-    const int launches = h->L * 2 + (h->use_tc ? 1 : 0);
+    const int launches = h->last_launches > 0 ? h->last_launches : h->L * 2 + (h->use_tc ? 1 : 0);
     const int64_t vals[9] = {h->sm_count, h->ncta_dir, h->threads, (int64_t)shp.smem, rows_res, rows_str,
                              (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches};
     for (int i = 0; i < n && i < 9; ++i) out[i] = vals[i];
