@@ -257,8 +257,10 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
     const int b_mine = vidx % BT;           // its batch row inside the chunk
     const int b_gather = lane & (BT - 1);   // batch row a lane < BT finalises
 
+#pragma unroll 1
     for (int s = 0; s < T; ++s) {
         const int t = d ? (T - 1 - s) : s;
+#pragma unroll 1
         for (int ci = 0; ci < nchunk; ++ci) {
             const int b0 = ci * BT;
             const int nb = min(BT, B - b0);
@@ -322,24 +324,23 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
             }
 
             // ---- gates and state update, one unit per warp at a time
+#pragma unroll 1
             for (int u = warp; u < nu; u += nwarps) {
                 AT acc[V];
 #pragma unroll
                 for (int i = 0; i < V; ++i) acc[i] = (AT)0;
                 if (!CSR) {
-                    if (u < units_res)
-                        unit_dot_dense<WT, BT, AT>(reinterpret_cast<const WT *>(res_base) + (size_t)u * 4 * a.Hp8,
-                                               a.Hp8, hb, Hs, lane, acc);
-                    else
-                        unit_dot_dense<WT, BT, AT>(wg + (size_t)u * 4 * a.Hp8, a.Hp8, hb, Hs, lane, acc);
+                    // one copy of the loop serves resident (shared) and streamed (global) units: the
+                    // base pointer is warp-uniform and the loads are generic
+                    const WT *rows = (u < units_res) ? reinterpret_cast<const WT *>(res_base) + (size_t)u * 4 * a.Hp8
+                                                     : wg + (size_t)u * 4 * a.Hp8;
+                    unit_dot_dense<WT, BT, AT>(rows, a.Hp8, hb, Hs, lane, acc);
                 } else {
                     int e[5];
 #pragma unroll
                     for (int i = 0; i < 5; ++i) e[i] = rp_s[4 * u + i] - ent_base;
-                    if (u < units_res)
-                        unit_dot_csr<ET, BT, AT>(reinterpret_cast<const ET *>(res_base), e, hb, Hs, lane, acc);
-                    else
-                        unit_dot_csr<ET, BT, AT>(eg + ent_base, e, hb, Hs, lane, acc);
+                    const ET *ents = (u < units_res) ? reinterpret_cast<const ET *>(res_base) : eg + ent_base;
+                    unit_dot_csr<ET, BT, AT>(ents, e, hb, Hs, lane, acc);
                 }
                 AT z = warp_reduce_multi<V, AT>(acc, lane);
 
