@@ -47,8 +47,9 @@ typedef struct lstm_handle lstm_handle;      /* opaque, library-owned */
 enum {
     LSTM_F32       = 0,   /* fp32 weights, fp32 activations and state, fp32 accumulation              */
     LSTM_BF16W_F32S = 1   /* weights rounded to bf16 (nearest-even) at create time; the input
-                             projection also rounds its activations to bf16 (tensor-core operands);
-                             state, accumulation, gates and outputs are fp32                            */
+                             projection feeds the tensor cores with each activation as two bf16
+                             terms (hi + lo, about 16 mantissa bits); state, accumulation, gates and
+                             outputs are fp32                                                           */
 };
 
 /* return codes */

@@ -293,7 +293,7 @@ bool want_tc(const lstm_handle *h)
 {
     if (h->dtype != LSTM_BF16W_F32S || h->exec_mode != LSTM_DENSE) return false;
     const char *env = getenv("LSTM_B200_PROJ");
-    return env && strcmp(env, "tc") == 0;
+    return !(env && strcmp(env, "simt") == 0);     // LSTM_B200_PROJ=simt selects the CUDA-core projection
 }
 
 int n_split_cap() { return 4; }
@@ -473,10 +473,10 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     rc = dev_alloc(h, &h->G, h->G_cap * 4, false, st, "projection workspace");
     if (rc == LSTM_OK && h->use_tc) {
         h->ld0 = round_up(in_dim, 8);
-        rc = dev_alloc(h, &h->xb0, Mmax * h->ld0 * 2, true, st, "bf16 input staging");
+        rc = dev_alloc(h, &h->xb0, 2 * Mmax * h->ld0 * 2, true, st, "bf16 input staging");
         if (rc == LSTM_OK && layers > 1) {
             h->ldn = round_up(D * H, 8);
-            for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->xbn[i], Mmax * h->ldn * 2, true, st, "bf16 layer activations");
+            for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->xbn[i], 2 * Mmax * h->ldn * 2, true, st, "bf16 layer activations");
         }
     }
     if (rc == LSTM_OK && layers > 1)
@@ -562,14 +562,15 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             __nv_bfloat16 *xb = l == 0 ? h->xb0 : h->xbn[(l - 1) & 1];
             if (l == 0) {
                 if (record(h, LSTM_K_STAGE, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-                e = launch_stage_bf16(x, xb, M, h->in_dim, h->ld0, st);
+                e = launch_stage_bf16(x, xb, (long long)h->max_T * h->max_B * h->ld0, M, h->in_dim, h->ld0, st);
                 ++h->last_launches;
                 if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
                 if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "staging launch failed: %s", cudaGetErrorString(e));
             }
             if (ly.plan_M != M) {
                 char msg[256];
-                if (proj_tc_plan(&ly.plan, (const __nv_bfloat16 *)ly.wx, xb, M, N, ly.in_l, ly.ldk, h->sm_count, msg, sizeof msg))
+                const long long plane = (long long)h->max_T * h->max_B * ly.ldk;
+                if (proj_tc_plan(&ly.plan, (const __nv_bfloat16 *)ly.wx, xb, xb + plane, M, N, ly.in_l, ly.ldk, h->sm_count, msg, sizeof msg))
                     return fail(h, LSTM_ERR_CUDA, "tensor-core projection plan failed: %s", msg);
                 ly.plan_M = M;
             }
@@ -605,6 +606,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         a.y = l == L - 1 ? y : h->ybuf[l & 1];
         a.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
         a.xb_ld = h->ldn;
+        a.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
         a.xch = h->xch;
         a.status = h->status_dev;
         if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");

@@ -37,8 +37,9 @@ struct RecurArgs {
     const float *h0, *c0;       // [D][B][H] of this layer or nullptr
     float *hT, *cT;             // [D][B][H] of this layer or nullptr
     float *y;                   // [T][B][D*H]
-    __nv_bfloat16 *xb_next;     // bf16 copy of y for the next layer's projection, or nullptr
-    int xb_ld;                  // its row stride in elements
+    __nv_bfloat16 *xb_next;     // y as two bf16 terms (hi plane, then lo plane) for the next layer's
+    long long xb_plane;         //   tensor-core projection, or nullptr; elements between the planes
+    int xb_ld;                  // row stride in elements
     unsigned long long *xch;    // [D][2][B][H] exchange words {stamp:32 | h bits:32}
     int *status;                // device status word
 };
@@ -53,8 +54,9 @@ cudaError_t recur_csr_prepare(int max_smem);
 // ---------------------------------------------------------------------------------------------------
 // Input staging and projection
 // ---------------------------------------------------------------------------------------------------
-// x fp32 [M][K] -> xb bf16 [M][ld] (columns K..ld-1 are written as zero)
-cudaError_t launch_stage_bf16(const float *x, __nv_bfloat16 *xb, long long M, int K, int ld,
+// x fp32 [M][K] -> two bf16 planes [M][ld]: hi = bf16(x), lo = bf16(x - hi) at xb + plane
+// (columns K..ld-1 are written as zero)
+cudaError_t launch_stage_bf16(const float *x, __nv_bfloat16 *xb, long long plane, long long M, int K, int ld,
                               cudaStream_t st);
 
 // G[m][n] = sum_k X[m][k] * W[n][k] + bias[n];  X fp32 [M][K], W [N][ldw] fp32 or bf16, G fp32 [M][N]
@@ -67,17 +69,18 @@ cudaError_t launch_proj_csr(const float *X, const int *rowptr, const CsrEntry *e
                             const float *bias, float *G, int M, int N, int K, bool f64_acc, cudaStream_t st);
 
 // Tensor-core projection (tcgen05 + TMEM + TMA).  A = packed weights [N][ldk] bf16 (K-major),
-// Bm = activations [M][ldk] bf16; writes G[split][M][N] fp32 (+bias on split 0).
+// activations [M][ldk] as two bf16 planes (hi, lo); writes G[split][M][N] fp32 (+bias on split 0).
 struct ProjTcPlan {
     alignas(64) unsigned char tmap_w[128];
     alignas(64) unsigned char tmap_x[128];
+    alignas(64) unsigned char tmap_xlo[128];
     int M, N, K, ldk;
     int n_tile;        // MMA N extent (activation rows per tile), multiple of 16, <= 256
     int nsplit;        // split-K factor
     int kblocks;       // ceil(K / 64)
 };
-int  proj_tc_plan(ProjTcPlan *p, const __nv_bfloat16 *W, const __nv_bfloat16 *X, int M, int N, int K,
-                  int ldk, int sm_count, char *err, int errlen);
+int  proj_tc_plan(ProjTcPlan *p, const __nv_bfloat16 *W, const __nv_bfloat16 *X, const __nv_bfloat16 *Xlo,
+                  int M, int N, int K, int ldk, int sm_count, char *err, int errlen);
 cudaError_t launch_proj_tc(const ProjTcPlan &p, const float *bias, float *G, int *status,
                            cudaStream_t st);
 cudaError_t proj_tc_prepare();

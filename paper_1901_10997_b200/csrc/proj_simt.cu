@@ -7,7 +7,7 @@
 namespace lstm {
 namespace {
 
-__global__ void stage_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__restrict__ xb,
+__global__ void stage_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__restrict__ xb, long long plane,
                                   long long M, int K, int ld)
 {
     const long long total = M * (long long)ld;
@@ -15,7 +15,10 @@ __global__ void stage_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__
          i += (long long)gridDim.x * blockDim.x) {
         const long long m = i / ld;
         const int k = (int)(i - m * ld);
-        xb[i] = __float2bfloat16_rn(k < K ? x[m * K + k] : 0.0f);
+        const float v = k < K ? x[m * K + k] : 0.0f;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        xb[i] = hi;
+        xb[plane + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
 }
 
@@ -125,14 +128,15 @@ __global__ void __launch_bounds__(256) proj_csr_kernel(const float *__restrict__
 
 }  // namespace
 
-cudaError_t launch_stage_bf16(const float *x, __nv_bfloat16 *xb, long long M, int K, int ld, cudaStream_t st)
+cudaError_t launch_stage_bf16(const float *x, __nv_bfloat16 *xb, long long plane, long long M, int K, int ld,
+                              cudaStream_t st)
 {
     const long long total = M * (long long)ld;
     if (total == 0) return cudaSuccess;
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
     if (blocks > 148LL * 8) blocks = 148LL * 8;
-    stage_bf16_kernel<<<(int)blocks, threads, 0, st>>>(x, xb, M, K, ld);
+    stage_bf16_kernel<<<(int)blocks, threads, 0, st>>>(x, xb, plane, M, K, ld);
     return cudaGetLastError();
 }
 

@@ -1,12 +1,325 @@
-// Tensor-core input projection (placeholder until the tcgen05 kernel lands).
+// Tensor-core input projection for bf16 storage: G[m][n] = sum_k X[m][k] Wx[n][k] (+ bias[n]), the x_t
+// half of W [x_t, h_{t-1}] + b of the paper's Section 4 cell equations for all timesteps at once.
+//
+// Blackwell-native structure: one CTA per (128 weight rows) x (n_tile activation rows) x (K split)
+// output tile.  Both operands are K-major bf16 and arrive through TMA (cp.async.bulk.tensor, 128-byte
+// swizzle, out-of-bounds rows and the K tail zero-filled) into a multi-stage shared-memory ring guarded
+// by mbarriers; one elected thread issues tcgen05.mma (M = 128, N = n_tile, K = 16 per instruction)
+// accumulating in tensor memory; four warps read the accumulator back with tcgen05.ld and store it with
+// the bias.  Activations are fed as two bf16 terms (x = hi + lo, lo = bf16(x - hi)): each weight tile
+// staged in shared memory is multiplied by both, so activations keep about 16 mantissa bits while the
+// weights -- exactly bf16 -- are read only once.  The weights are the M operand, so a short sequence
+// (T*B = 35) still fills the MMA's 128-row dimension; such weight-read-bound shapes are split along K
+// over otherwise idle SMs and the partial planes are added up by the recurrent kernel.  No TMA multicast is used: each CTA fetches its
+// own tiles.  Every mbarrier wait is bounded; on expiry the kernel records a timeout status, and all
+// roles fall through to the common exit where tensor memory is released.
 #include "common.cuh"
+
+#include <cuda.h>
 #include <cstdio>
+#include <cstring>
+
 namespace lstm {
-int proj_tc_plan(ProjTcPlan *, const __nv_bfloat16 *, const __nv_bfloat16 *, int, int, int, int, int, char *err, int errlen)
+namespace {
+
+constexpr int kBM = 128;          // weight rows per tile (MMA M)
+constexpr int kBK = 64;           // K elements per stage: 128 bytes of bf16 = one swizzle atom row
+constexpr int kThreads = 192;     // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
+constexpr int kMaxStages = 8;
+constexpr int kMaxNTile = 128;    // activation rows per tile (MMA N); two activation tiles (hi, lo) per stage
+constexpr long long kWaitLimit = 1ll << 24;   // try_wait attempts before a wait gives up
+
+struct TcArgs {
+    int M, N, K;
+    int n_tile, nsplit, kblocks, stages, tmem_cols;
+    float *G;
+    const float *bias;
+    int *status;
+    long long g_split_stride;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    snprintf(err, errlen, "tensor-core projection not built");
-    return 1;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-cudaError_t launch_proj_tc(const ProjTcPlan &, const float *, float *, int *, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t proj_tc_prepare() { return cudaSuccess; }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when it gave up (or another role did): the caller leaves its loop.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (long long it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255) == 255 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+// K-major operand tile in shared memory, 128-byte swizzle: rows of 128 bytes, groups of 8 rows are
+// 1024 bytes apart (stride byte offset); version field = 1 for this architecture.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);          // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                                 // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                       // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                                 // descriptor version
+    d |= (uint64_t)2 << 61;                                 // layout type: 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+proj_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+               const __grid_constant__ CUtensorMap tmap_xlo, const TcArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ __align__(8) unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int w_tile = blockIdx.x, x_tile = blockIdx.y, split = blockIdx.z;
+    const int kb0 = (int)((long long)split * a.kblocks / a.nsplit);
+    const int kb1 = (int)((long long)(split + 1) * a.kblocks / a.nsplit);
+    const int nkb = kb1 - kb0;
+    const int S = a.stages;
+    const uint32_t a_bytes = kBM * kBK * 2, b_bytes = (uint32_t)a.n_tile * kBK * 2;
+    const uint32_t stage_bytes = a_bytes + 2 * b_bytes;                 // weights, x hi, x lo; multiple of 1024
+    const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;      // swizzled tiles need 1024-byte alignment
+
+    if (tid == 0) {
+        abort_s = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        mbar_init(smem_u32(&accum_bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_s;
+    volatile int *abort_flag = &abort_s;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % S;
+                const uint32_t ph = (uint32_t)(i / S) & 1u;
+                if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) break;
+                const uint32_t fb = smem_u32(&full_bar[s]);
+                mbar_expect_tx(fb, stage_bytes);
+                const uint32_t sa = tiles + (uint32_t)s * stage_bytes;
+                tma_load_2d(sa, &tmap_w, fb, (kb0 + i) * kBK, w_tile * kBM);
+                tma_load_2d(sa + a_bytes, &tmap_x, fb, (kb0 + i) * kBK, x_tile * a.n_tile);
+                tma_load_2d(sa + a_bytes + b_bytes, &tmap_xlo, fb, (kb0 + i) * kBK, x_tile * a.n_tile);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = n_tile, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.n_tile >> 3) << 17) |
+                                   ((uint32_t)(kBM >> 4) << 24);
+            bool ok = true;
+            for (int i = 0; i < nkb && ok; ++i) {
+                const int s = i % S;
+                const uint32_t ph = (uint32_t)(i / S) & 1u;
+                ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = tiles + (uint32_t)s * stage_bytes;
+#pragma unroll
+                for (int k = 0; k < kBK / 16; ++k) {
+                    const uint64_t adesc = umma_desc_sw128(sa + k * 32);
+                    const uint64_t bhi = umma_desc_sw128(sa + a_bytes + k * 32);
+                    const uint64_t blo = umma_desc_sw128(sa + a_bytes + b_bytes + k * 32);
+                    umma_bf16(tmem_base, adesc, bhi, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    umma_bf16(tmem_base, adesc, blo, idesc, 1u);
+                }
+                umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(smem_u32(&accum_bar));     // accumulator complete
+        }
+    } else {
+        // ---- epilogue: warp w may touch TMEM lanes 32*(w % 4) .. +31
+        const int lq = warp & 3;
+        const bool ok = mbar_wait(smem_u32(&accum_bar), 0u, abort_flag);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const int n = w_tile * kBM + lq * 32 + lane;                  // weight row = G column
+            const float bv = (split == 0 && a.bias && n < a.N) ? a.bias[n] : 0.0f;
+            float *gout = a.G + (size_t)split * a.g_split_stride;
+            for (int c0 = 0; c0 < a.n_tile; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const int m0 = x_tile * a.n_tile + c0;
+                if (n < a.N) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (m0 + i < a.M) gout[(size_t)(m0 + i) * a.N + n] = __uint_as_float(v[i]) + bv;
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+    }
+    if (tid == 0 && abort_s) atomicExch(a.status, kStatusTimeout);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// rows x K bf16 matrix with row stride ldk elements; box = 64 x box_rows, 128-byte swizzle, zero fill
+bool encode_2d(CUtensorMap *map, const void *base, int rows, int K, int ldk, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldk * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kSmemBudget = 200 * 1024;
+
+}  // namespace
+
+static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+
+int proj_tc_plan(ProjTcPlan *p, const __nv_bfloat16 *W, const __nv_bfloat16 *X, const __nv_bfloat16 *Xlo,
+                 int M, int N, int K, int ldk, int sm_count, char *err, int errlen)
+{
+    if (M < 1 || N < 1 || K < 1 || (ldk % 8) != 0 || ((uintptr_t)W & 15) || ((uintptr_t)X & 15) || ((uintptr_t)Xlo & 15)) {
+        snprintf(err, errlen, "operands must be 16-byte aligned with row strides that are multiples of 8 elements");
+        return 1;
+    }
+    memset(p, 0, sizeof *p);
+    p->M = M; p->N = N; p->K = K; p->ldk = ldk;
+    p->kblocks = (K + kBK - 1) / kBK;
+    const int wtiles = (N + kBM - 1) / kBM;
+    int xtiles = (M + kMaxNTile - 1) / kMaxNTile;
+    int n_tile = ((M + xtiles - 1) / xtiles + 15) / 16 * 16;
+    if (n_tile > kMaxNTile) n_tile = kMaxNTile;
+    xtiles = (M + n_tile - 1) / n_tile;
+    p->n_tile = n_tile;
+    // weight-read-bound shapes (a single activation tile): split K over SMs that would otherwise idle
+    int nsplit = 1;
+    if (xtiles == 1) {
+        nsplit = sm_count / wtiles;
+        if (nsplit > 4) nsplit = 4;
+        if (nsplit > p->kblocks) nsplit = p->kblocks;
+        if (nsplit < 1) nsplit = 1;
+    }
+    p->nsplit = nsplit;
+    if (!encode_2d(reinterpret_cast<CUtensorMap *>(p->tmap_w), W, N, K, ldk, kBM) ||
+        !encode_2d(reinterpret_cast<CUtensorMap *>(p->tmap_x), X, M, K, ldk, n_tile) ||
+        !encode_2d(reinterpret_cast<CUtensorMap *>(p->tmap_xlo), Xlo, M, K, ldk, n_tile)) {
+        snprintf(err, errlen, "cuTensorMapEncodeTiled failed (N=%d M=%d K=%d ldk=%d n_tile=%d)", N, M, K, ldk, n_tile);
+        return 1;
+    }
+    return 0;
+}
+
+cudaError_t proj_tc_prepare()
+{
+    return cudaFuncSetAttribute(proj_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024);
+}
+
+cudaError_t launch_proj_tc(const ProjTcPlan &p, const float *bias, float *G, int *status, cudaStream_t st)
+{
+    TcArgs a;
+    a.M = p.M; a.N = p.N; a.K = p.K;
+    a.n_tile = p.n_tile; a.nsplit = p.nsplit; a.kblocks = p.kblocks;
+    const int stage_bytes = kBM * kBK * 2 + 2 * p.n_tile * kBK * 2;
+    int stages = kSmemBudget / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    const int max_kb = (p.kblocks + p.nsplit - 1) / p.nsplit;
+    if (stages > max_kb) stages = max_kb;
+    if (stages < 1) stages = 1;
+    a.stages = stages;
+    int cols = 32;
+    while (cols < p.n_tile) cols <<= 1;
+    a.tmem_cols = cols;
+    a.G = G; a.bias = bias; a.status = status;
+    a.g_split_stride = (long long)p.M * p.N;
+    const int wtiles = (p.N + kBM - 1) / kBM;
+    const int xtiles = (p.M + p.n_tile - 1) / p.n_tile;
+    dim3 grid(wtiles, xtiles, p.nsplit);
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    proj_tc_kernel<<<grid, kThreads, smem, st>>>(*reinterpret_cast<const CUtensorMap *>(p.tmap_w),
+                                                 *reinterpret_cast<const CUtensorMap *>(p.tmap_x),
+                                                 *reinterpret_cast<const CUtensorMap *>(p.tmap_xlo), a);
+    return cudaGetLastError();
+}
+
 }  // namespace lstm

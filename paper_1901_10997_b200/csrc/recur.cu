@@ -371,8 +371,12 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
                                        (unsigned long long)__float_as_uint(hn));
                     c_s[u * B + b] = cn;
                     a.y[((size_t)t * B + b) * D * H + (size_t)d * H + j] = hn;
-                    if (a.xb_next)
-                        a.xb_next[((size_t)t * B + b) * a.xb_ld + (size_t)d * H + j] = __float2bfloat16_rn(hn);
+                    if (a.xb_next) {
+                        const size_t xi = ((size_t)t * B + b) * a.xb_ld + (size_t)d * H + j;
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
+                        a.xb_next[xi] = hi;
+                        a.xb_next[a.xb_plane + xi] = __float2bfloat16_rn(hn - __bfloat162float(hi));
+                    }
                     if (s == T - 1) {
                         if (a.hT) a.hT[((size_t)d * B + b) * H + j] = hn;
                         if (a.cT) a.cT[((size_t)d * B + b) * H + j] = cn;
