@@ -172,6 +172,24 @@ def run_reference(args):
     }))
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (the slowest replica sets the job's
+    time); identity without a process group."""
+    import torch
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(world: int, seqs_per_replica: int, ms_per_step: float):
+    """Replicas only: every rank runs the same workload on its own sequences, so one step of the job
+    processes world * B sequences in the slowest rank's step time.  Returns (sequences per step,
+    microseconds per sequence, sequences per second)."""
+    seqs = world * seqs_per_replica
+    return seqs, ms_per_step * 1e3 / seqs, seqs / (ms_per_step * 1e-3)
+
+
 def flush_l2(buf):
     buf.zero_()
 
@@ -283,15 +301,11 @@ def run_gpu(args):
     e2e_total -= time.perf_counter() - t0
     barrier()
 
-    tot = torch.tensor([total_ms, e2e_total * 1e3], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(tot, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(tot[0]), float(tot[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_total * 1e3], dist, dev)
 
     if rank == 0:
         ms_per_step = total_ms / args.steps
-        seqs = world * w.B
-        us_per_seq = ms_per_step * 1e3 / seqs
+        seqs, us_per_seq, seqs_per_sec = job_throughput(world, w.B, ms_per_step)
         peak, peak_kind = measured_peaks()
         nnz = None
         if mode == "csr":
@@ -315,7 +329,7 @@ def run_gpu(args):
             "config": {"workload": w.name, "layers": w.layers, "dirs": w.dirs, "in_dim": w.in_dim, "hidden": w.hidden,
                        "T": w.T, "B": w.B, "exec_mode": mode, "weights": w.dtype, "state": "fp32", "l2": "flushed between timed steps (256 MiB write)",
                        "parallelism": f"replicas x{world}"},
-            "sequences_per_sec": seqs / (ms_per_step * 1e-3),
+            "sequences_per_sec": seqs_per_sec,
             "step_ms_p10_p50_p90": [float(np.percentile(ms, q)) for q in (10, 50, 90)],
             "clocks": clocks.summary(),
             "gpu_launches": int(launches_per_fwd * args.steps),
