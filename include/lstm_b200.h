@@ -154,6 +154,34 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 
+/*
+ * Forward pass without any allocation (the paper has no counterpart: this exists for deployment).
+ * For callers that cannot allocate device memory at call time or at all -- a serving loop whose memory
+ * pool is fixed at start-up, a host framework whose allocator owns the device, a process that must not
+ * grow after initialisation -- and therefore cannot use lstm_create, which allocates packed weights and
+ * a workspace.  One layer, one direction, fp32, dense; every tensor is the caller's:
+ *   wx [4H, in_dim], wh [4H, H] row-major fp32 and b [4H] (or NULL = zeros), gate row blocks i,f,g,o;
+ *   x [T,B,in_dim]; h0, c0 [B,H] or NULL (zeros); y [T,B,H]; hT, cT [B,H] or NULL (not wanted).
+ * All are DEVICE pointers and are only read (wx, wh, b, x, h0, c0) or written (y, hT, cT) by this call.
+ * The same cell equations as lstm_forward, fp32 accumulation; weights are read through L2 every step
+ * (nothing is packed or kept on-chip), so this path is slower than a handle.
+ * Scratch: the per-step exchange words and a status word live in a fixed array inside the library
+ * image (about 128 KiB of device memory on every GPU that loads the library, held until exit).
+ * Limits: B * hidden <= LSTM_NOALLOC_MAX_BH and B * (in_dim + hidden + hidden/SMs + 1) floats must fit
+ * in one CTA's shared memory; beyond them the call returns LSTM_ERR_UNSUPPORTED and launches nothing.
+ * The first call on a device (with that device current) looks up the array's device address and the
+ * device limits; make that first call before any stream capture.  Every call clears the array and then
+ * uses it: calls that overlap on the same GPU (two streams, two threads) race on it and must be
+ * serialised by the caller.  The call calls no cudaMalloc / cudaFree or any allocating routine; it
+ * enqueues on cuda_stream and synchronises that stream before returning, so a device-side timeout of
+ * this very call is returned as LSTM_ERR_TIMEOUT.
+ * err (may be NULL): caller-owned buffer of errlen bytes that receives the reason of a failure.
+ */
+#define LSTM_NOALLOC_MAX_BH 8192
+LSTM_API int lstm_forward_noalloc(const float *wx, const float *wh, const float *b, int in_dim, int hidden,
+                         const float *x, int T, int B, const float *h0, const float *c0,
+                         float *y, float *hT, float *cT, void *cuda_stream, char *err, int errlen);
+
 #ifdef __cplusplus
 }
 #endif

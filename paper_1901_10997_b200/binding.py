@@ -64,6 +64,8 @@ def load_library():
         lib.lstm_profile_read.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ctypes.c_float)]
         lib.lstm_info.restype = ci
         lib.lstm_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), ci]
+        lib.lstm_forward_noalloc.restype = ci
+        lib.lstm_forward_noalloc.argtypes = [vp, vp, vp, ci, ci, vp, ci, ci, vp, vp, vp, vp, vp, vp, ctypes.c_char_p, ci]
         _lib = lib
     return _lib
 
@@ -117,6 +119,17 @@ def lstm_info(handle):
     keys = ["sm_count", "ctas_per_dir", "threads", "smem_bytes", "rows_resident", "rows_streamed",
             "proj_splits", "proj_tensor_core", "launches_per_forward"]
     return {k: int(out[i]) for i, k in enumerate(keys[:n])}
+
+
+def lstm_forward_noalloc(wx, wh, b, in_dim, hidden, x, T, B, h0, c0, y, hT, cT, stream=0):
+    """One fp32 layer straight from the caller's device buffers (addresses as integers), using only
+    the scratch array built into the library: for callers that may not allocate device memory.
+    Returns (code, message)."""
+    err = ctypes.create_string_buffer(512)
+    rc = load_library().lstm_forward_noalloc(wx or None, wh or None, b or None, in_dim, hidden, x or None, T, B,
+                                             h0 or None, c0 or None, y or None, hT or None, cT or None,
+                                             stream or None, err, len(err))
+    return rc, err.value.decode()
 
 
 # ---------------------------------------------------------------- convenience wrapper
