@@ -150,7 +150,9 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
  * [2] threads per CTA, [3] dynamic shared memory bytes per CTA at max_B, [4] recurrent-matrix rows
  * resident in shared memory per CTA (max over CTAs), [5] rows streamed from L2 per CTA (max),
  * [6] split-K factor of the input projection at max_T*max_B, [7] 1 if the projection uses the tensor-core
- * (tcgen05) kernel, [8] kernels launched by the most recent lstm_forward (before the first call: the count expected).
+ * (tcgen05) kernel, [8] kernels launched by the most recent lstm_forward (before the first call: the count expected),
+ * [9] 1 if the recurrence keeps its weights in registers (bf16 dense), 0 for the shared-memory kernel,
+ * [10] 16-column weight tiles per warp held in registers, [11] per warp held in shared memory.
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 

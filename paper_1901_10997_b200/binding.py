@@ -117,7 +117,8 @@ def lstm_info(handle):
     out = (ctypes.c_int64 * 16)()
     n = load_library().lstm_info(handle, out, 16)
     keys = ["sm_count", "ctas_per_dir", "threads", "smem_bytes", "rows_resident", "rows_streamed",
-            "proj_splits", "proj_tensor_core", "launches_per_forward"]
+            "proj_splits", "proj_tensor_core", "launches_per_forward", "recur_register_resident",
+            "col_tiles_in_registers", "col_tiles_in_smem"]
     return {k: int(out[i]) for i, k in enumerate(keys[:n])}
 
 

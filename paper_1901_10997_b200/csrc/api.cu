@@ -29,6 +29,7 @@ struct Layer {
     void *wh[2] = {nullptr, nullptr};  // dense [H][4][Hp8]
     int *wh_ptr[2] = {nullptr, nullptr};   // CSR recurrence: padded entry offsets [4H+1]
     void *wh_ent[2] = {nullptr, nullptr};
+    uint4 *wfrag[2] = {nullptr, nullptr};  // register-resident kernel: operand-A fragments
     int csr_max_slice_entries = 0;     // largest per-CTA slice (entries, padded)
     ProjTcPlan plan;                   // tensor-core projection plan for plan_M rows
     int plan_M = -1;
@@ -42,6 +43,10 @@ struct lstm_handle {
     int Hp8 = 0, Hs = 0;
     int ncta_dir = 0, upc = 0, threads = 0;
     bool use_tc = false;
+    // register-resident recurrent kernel (bf16 dense): row tiles, column tiles per warp in registers and
+    // in shared memory, warps per CTA
+    bool use_mma = false;
+    int mma_mt = 0, mma_nkr = 0, mma_nks = 0, mma_nw = 0;
     std::vector<Layer> layers;
     // workspace
     float *G = nullptr; size_t G_cap = 0;
@@ -231,6 +236,14 @@ struct RecurShape { int BT; size_t smem; int w_smem_bytes; int units_res_min; };
 
 RecurShape recur_shape(const lstm_handle *h, int B, int layer)
 {
+    if (h->use_mma) {
+        RecurShape s;
+        s.BT = 4;
+        s.smem = recur_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc, B);
+        s.w_smem_bytes = h->mma_nw * h->mma_nks * h->mma_mt * 512;
+        s.units_res_min = 0;
+        return s;
+    }
     const size_t budget = (size_t)h->smem_optin - 64;            // static shared memory of the kernel
     const bool csr = h->exec_mode == LSTM_CSR;
     const size_t wsize = h->dtype == LSTM_BF16W_F32S ? 2 : 4;
@@ -267,8 +280,35 @@ RecurShape recur_shape(const lstm_handle *h, int B, int layer)
     return s;
 }
 
+// Chooses the tiling of the register-resident recurrent kernel, or leaves use_mma false when the
+// slice of a CTA does not fit registers + shared memory (then the shared-memory kernel runs).
+void plan_mma(lstm_handle *h)
+{
+    h->use_mma = false;
+    if (h->dtype != LSTM_BF16W_F32S || h->exec_mode != LSTM_DENSE) return;
+    const char *env = getenv("LSTM_B200_RECUR");
+    if (env && strcmp(env, "simt") == 0) return;      // LSTM_B200_RECUR=simt selects the shared-memory kernel
+    const int mt = (4 * h->upc + 15) / 16;
+    if (mt > 4) return;
+    const int nk = (h->H + 15) / 16;
+    const int nw = (nk <= 32 && h->upc <= 8) ? 8 : 16;   // warp w also finishes unit w: upc <= warps
+    if (h->upc > nw) return;
+    const int need = (nk + nw - 1) / nw;               // column tiles per warp
+    const int cap = (nw == 16 ? kMmaTileCap16 : kMmaTileCap8) / mt;
+    int nkr = 0;
+    for (int c = 2; c <= 8; c += 2)
+        if (c <= cap && (nkr == 0 || nkr < need)) nkr = c;     // smallest even count >= need, else the largest allowed
+    if (nkr == 0) return;
+    const int nks = need > nkr ? need - nkr : 0;
+    if (!recur_mma_shape_ok(mt, nkr, nw)) return;
+    if (recur_mma_smem_bytes(mt, nkr, nw, nks, h->upc, h->max_B) > (size_t)h->smem_optin - 64) return;
+    h->use_mma = true;
+    h->mma_mt = mt; h->mma_nkr = nkr; h->mma_nks = nks; h->mma_nw = nw;
+}
+
 int max_b_fits(const lstm_handle *h)
 {
+    if (h->use_mma) return 1;
     // the staging buffers and the c state must fit even when no weight is resident
     const size_t budget = (size_t)h->smem_optin - 64;
     const size_t c_bytes = (size_t)round_up(h->upc * h->max_B, 4) * 4;
@@ -280,7 +320,7 @@ void free_all(lstm_handle *h)
 {
     for (auto &ly : h->layers) {
         cudaFree(ly.wx); cudaFree(ly.bias); cudaFree(ly.wx_rowptr); cudaFree(ly.wx_ent);
-        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); }
+        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); }
     }
     cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
     cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->status_dev);
@@ -345,6 +385,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
+    plan_mma(h);
     h->layers.resize(layers);
     if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
 
@@ -391,7 +432,34 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                 rc = matrix_to_dense(h, 4 * H, H, src.wh, src.mask_h, src.wh_rowptr, src.wh_col, src.wh_val, m, name);
                 if (rc) break;
                 const size_t n = (size_t)H * 4 * h->Hp8;
-                if (bf16) {
+                if (h->use_mma) {
+                    // operand-A fragments: [cta][warp][column tile][row tile][lane] x 4 words; local row
+                    // r = 4 * unit + gate, zero beyond the CTA's units and beyond column H
+                    const int NW = h->mma_nw, nkw = h->mma_nkr + h->mma_nks, MT = h->mma_mt;
+                    std::vector<uint32_t> f((size_t)h->ncta_dir * NW * nkw * MT * 32 * 4, 0u);
+                    size_t o = 0;
+                    for (int c = 0; c < h->ncta_dir; ++c) {
+                        int u0, nu; unit_range_host(H, h->ncta_dir, c, u0, nu);
+                        auto wv = [&](int r, int k) -> uint32_t {
+                            if (r >= 4 * nu || k >= H) return 0u;
+                            return f32_to_bf16_rne(m[(size_t)((r & 3) * H + u0 + (r >> 2)) * H + k]);
+                        };
+                        for (int wp = 0; wp < NW; ++wp)
+                            for (int i = 0; i < nkw; ++i)
+                                for (int mt = 0; mt < MT; ++mt)
+                                    for (int lane = 0; lane < 32; ++lane) {
+                                        const int g = lane >> 2, p2 = (lane & 3) * 2;
+                                        const int r0 = mt * 16 + g, r1 = r0 + 8;
+                                        const int ka = (wp * nkw + i) * 16 + p2, kb = ka + 8;
+                                        f[o++] = wv(r0, ka) | (wv(r0, ka + 1) << 16);
+                                        f[o++] = wv(r1, ka) | (wv(r1, ka + 1) << 16);
+                                        f[o++] = wv(r0, kb) | (wv(r0, kb + 1) << 16);
+                                        f[o++] = wv(r1, kb) | (wv(r1, kb + 1) << 16);
+                                    }
+                    }
+                    rc = upload(h, (uint32_t **)&ly.wfrag[d], f.data(), f.size() * 4, st, "recurrent weight fragments");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                } else if (bf16) {
                     std::vector<uint16_t> p(n, 0);
                     for (int j = 0; j < H; ++j)
                         for (int q = 0; q < 4; ++q) {
@@ -485,7 +553,9 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->xch, h->xch_words * 8, true, st, "exchange buffer");
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
     if (rc == LSTM_OK) {
-        cudaError_t e = csr ? recur_csr_prepare(h->smem_optin - 64) : recur_dense_prepare(h->smem_optin - 64);
+        cudaError_t e = csr ? recur_csr_prepare(h->smem_optin - 64)
+                            : h->use_mma ? recur_mma_prepare(h->mma_mt, h->mma_nkr, h->mma_nw, h->smem_optin - 64)
+                                         : recur_dense_prepare(h->smem_optin - 64);
         if (e == cudaSuccess && h->use_tc) e = proj_tc_prepare();
         if (e != cudaSuccess) rc = fail(h, LSTM_ERR_CUDA, "kernel set-up failed: %s", cudaGetErrorString(e));
     }
@@ -590,6 +660,32 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
 
         // ---- recurrence
         const RecurShape shp = recur_shape(h, B, l);
+        if (h->use_mma) {
+            RecurMmaArgs m;
+            memset(&m, 0, sizeof m);
+            m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit; m.nkw_smem = h->mma_nks;
+            m.stamp_base = h->stamp_next;
+            h->stamp_next += (unsigned)T + 1u;
+            m.spin_limit = h->spin_limit;
+            for (int d = 0; d < D; ++d) m.wfrag[d] = ly.wfrag[d];
+            m.G = h->G;
+            m.g_split_stride = (long long)M * N;
+            const size_t so = (size_t)l * D * B * H;
+            m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
+            m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
+            m.y = l == L - 1 ? y : h->ybuf[l & 1];
+            m.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
+            m.xb_ld = h->ldn;
+            m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
+            m.xch = h->xch;
+            m.status = h->status_dev;
+            if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_recur_mma(m, h->mma_mt, h->mma_nkr, h->mma_nw, shp.smem, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
+            continue;
+        }
         RecurArgs a;
         memset(&a, 0, sizeof a);
         a.H = H; a.Hp8 = h->Hp8; a.Hs = h->Hs; a.B = B; a.T = T; a.D = D;
@@ -709,17 +805,20 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
     const RecurShape shp = recur_shape(h, h->max_B, 0);
     const size_t wsize = h->dtype == LSTM_BF16W_F32S ? 2 : 4;
     int64_t rows_res = 0, rows_str = 0;
-    if (h->exec_mode == LSTM_DENSE) {
+    if (h->use_mma) {
+        rows_res = 4 * h->upc;
+    } else if (h->exec_mode == LSTM_DENSE) {
         const size_t unit_bytes = (size_t)4 * h->Hp8 * wsize;
         const int ures = (int)std::min<size_t>(h->upc, shp.w_smem_bytes / unit_bytes);
         rows_res = 4 * ures; rows_str = 4 * (h->upc - ures);
     }
     const Layer &l0 = h->layers[0];
     const int launches = h->last_launches > 0 ? h->last_launches : h->L * 2 + (h->use_tc ? 1 : 0);
-    const int64_t vals[9] = {h->sm_count, h->ncta_dir, h->threads, (int64_t)shp.smem, rows_res, rows_str,
-                             (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches};
-    for (int i = 0; i < n && i < 9; ++i) out[i] = vals[i];
-    return 9;
+    const int64_t vals[12] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->threads, (int64_t)shp.smem,
+                              rows_res, rows_str, (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches,
+                              h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0};
+    for (int i = 0; i < n && i < 12; ++i) out[i] = vals[i];
+    return 12;
 }
 
 }  // extern "C"

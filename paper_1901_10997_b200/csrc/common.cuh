@@ -52,6 +52,40 @@ cudaError_t recur_dense_prepare(int max_smem);   // raises the dynamic shared-me
 cudaError_t recur_csr_prepare(int max_smem);
 
 // ---------------------------------------------------------------------------------------------------
+// Register-resident recurrent kernel (bf16 weights, dense).  Same CTA/unit partition and exchange
+// buffer as above.  The slice of a CTA is cut into 16 x 16 tiles: MT row tiles (4 gate rows per unit,
+// zero-padded) by NW * nkw column tiles; warp w owns column tiles [w * nkw, (w + 1) * nkw) of every row
+// tile, the first NKR of them in registers, the remaining nkw_smem in shared memory.
+// ---------------------------------------------------------------------------------------------------
+struct RecurMmaArgs {
+    int H, B, T, D;
+    int ncta_dir;
+    int nsplit;
+    int nkw_smem;               // trailing column tiles of every warp kept in shared memory
+    unsigned stamp_base;
+    long long spin_limit;
+    // per direction [cta][warp][column tile][row tile][lane] 16-byte operand-A fragments:
+    // lane (g = lane / 4, p = lane % 4) holds rows g and g + 8, columns 2p, 2p+1 and 2p+8, 2p+9
+    const uint4 *wfrag[2];
+    const float *G;
+    long long g_split_stride;
+    const float *h0, *c0;
+    float *hT, *cT;
+    float *y;
+    __nv_bfloat16 *xb_next;
+    long long xb_plane;
+    int xb_ld;
+    unsigned long long *xch;
+    int *status;
+};
+constexpr int kMmaTileCap16 = 18;   // MT * NKR limit with 16 warps (128 registers per thread, no spills)
+constexpr int kMmaTileCap8 = 40;    // ... with 8 warps
+bool recur_mma_shape_ok(int mt, int nkr, int nw);
+size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B);
+cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
+cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------
 // Input staging and projection
 // ---------------------------------------------------------------------------------------------------
 // x fp32 [M][K] -> two bf16 planes [M][ld]: hi = bf16(x), lo = bf16(x - hi) at xb + plane
