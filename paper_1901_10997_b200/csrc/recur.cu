@@ -35,6 +35,14 @@ __device__ __forceinline__ int ld_volatile_s32(const int *p)
     return v;
 }
 
+// read-only load that the compiler may not sink towards its use: issued before a wait, consumed after it
+__device__ __forceinline__ float ld_nc_early(const float *p)
+{
+    float v;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
 __device__ __forceinline__ float sigmoid_f(float z) { return 1.0f / (1.0f + expf(-z)); }
 
 // Position of hidden index k inside a staged h row.  Dense kernels read eight consecutive h values
@@ -267,11 +275,14 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
             float *hb = h_s + (size_t)((s * nchunk + ci) & 1) * BT * Hs;
 
             // projection term of this warp's first unit, fetched before the wait
-            float g_pre = 0.0f;
+            // (one register per split-K plane, added up only after the wait, so the loads stay in flight)
+            float g_pl[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (warp < nu && b_mine < nb) {
                 const float *gp = a.G + (((size_t)t * B + b0 + b_mine) * D + d) * 4 * H +
                                   (size_t)(u0 + warp) * 4 + q_mine;
-                for (int sp = 0; sp < a.nsplit; ++sp) g_pre += __ldg(gp + (size_t)sp * a.g_split_stride);
+#pragma unroll
+                for (int sp = 0; sp < 4; ++sp)
+                    if (sp < a.nsplit) g_pl[sp] = ld_nc_early(gp + (size_t)sp * a.g_split_stride);
             }
 
             // ---- stage h_{t-1} rows b0 .. b0+nb-1 into shared memory
@@ -344,7 +355,7 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
                 }
                 AT z = warp_reduce_multi<V, AT>(acc, lane);
 
-                float g_in = g_pre;
+                float g_in = (g_pl[0] + g_pl[1]) + (g_pl[2] + g_pl[3]);
                 if (u != warp) {
                     g_in = 0.0f;
                     if (b_mine < nb) {
@@ -383,6 +394,10 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
                     }
                 }
             }
+            // Pacing: no warp starts to poll for the next pass before this CTA has issued its own stores;
+            // loads that spin on words that are not there yet would sit in front of those stores on the
+            // way to L2 and delay every other CTA.
+            __syncthreads();
         }
     }
 }
