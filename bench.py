@@ -63,6 +63,24 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_traffic(kernel: str, workload: str, source: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary
+    profiles/<kernel>_<workload>.md, or None when there is none or the kernel's source has changed since
+    the counters were taken (the summary records the sha256 of the source file it profiled)."""
+    import hashlib
+    import re
+    f = ROOT / "profiles" / f"{kernel}_{workload}.md"
+    src = ROOT / "paper_1901_10997_b200" / "csrc" / source
+    if not (f.exists() and src.exists()):
+        return None
+    text = f.read_text()
+    m_sha = re.search(r"source_sha256:\s*([0-9a-f]{64})", text)
+    m_tr = re.search(r"traffic_bytes_per_launch:\s*([0-9]+)", text)
+    if not (m_sha and m_tr) or hashlib.sha256(src.read_bytes()).hexdigest() != m_sha.group(1):
+        return None
+    return int(m_tr.group(1))
+
+
 def recurrence_bytes_per_launch(w: wl.Workload, nnz_per_layer=None) -> float:
     """Algorithmic bytes one recurrent-kernel launch (one layer, all T steps, all directions) needs if
     nothing were resident: per step and direction the recurrent matrix once (4H*H*w bytes dense, or
@@ -314,13 +332,10 @@ def run_gpu(args):
         alg_bytes = recurrence_bytes_per_launch(w, nnz)
         rec_avg_ms = rec_ms / max(rec_n, 1)
         achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
-        traffic = None
-        tp = ROOT / "profiles" / "traffic.json"
-        if tp.exists():
-            try:
-                traffic = json.loads(tp.read_text()).get(f"recur/{args.workload}")
-            except Exception:
-                traffic = None
+        info = model.info()
+        kernel_name, kernel_src = (("recur_mma_kernel", "recur_mma.cu") if info.get("recur_register_resident")
+                                   else ("recur_kernel", "recur.cu"))
+        traffic = measured_traffic(kernel_name, args.workload, kernel_src)
         line = {
             "metric": "us_per_sequence", "value": us_per_seq, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
@@ -336,14 +351,14 @@ def run_gpu(args):
             "e2e": {"value": e2e_ms * 1e3 / e2e_steps / seqs, "unit": "us",
                     "h2d_bytes_per_step": int(x.nbytes),
                     "d2h_bytes_per_step": int(yh.numel() * 4 + hTh.numel() * 4 + cTh.numel() * 4)},
-            "roofline": {"bound": "hbm", "kernel": "recur_kernel (one launch = one layer, all T steps)",
+            "roofline": {"bound": "hbm", "kernel": f"{kernel_name} (one launch = one layer, all T steps)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": (achieved / peak if achieved else None), "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
                          "avg_launch_ms": rec_avg_ms,
                          "us_per_timestep": rec_avg_ms * 1e3 / w.T,
-                         "note": "weights are resident in shared memory, so the fraction of the HBM "
-                                 "weight-read bound may exceed 1"},
+                         "note": "the recurrent matrix stays on-chip (registers / shared memory) for the whole "
+                                 "sequence, so the fraction of the per-step HBM weight-read bound may exceed 1"},
             "kernel_ms_per_forward": {"stage": stage_ms / args.steps, "projection": proj_ms / args.steps,
                                       "recurrence": rec_ms / args.steps},
             "library": model.info(),
