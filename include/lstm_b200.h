@@ -135,6 +135,16 @@ LSTM_API int lstm_destroy(lstm_handle *h);
 LSTM_API const char *lstm_last_error(const lstm_handle *h);
 
 /*
+ * Failure-path self-test.  The recurrent kernels hand h_t from CTA to CTA through stamped words and
+ * every wait for such a word is bounded.  With cta >= 0, the recurrent kernel's CTA of that index
+ * withholds its words in the following lstm_forward calls, so the waits of the other CTAs run out after
+ * spin_limit clock ticks (spin_limit <= 0: the default limit, about a second): the kernel records
+ * LSTM_ERR_TIMEOUT, stops waiting and runs to its end, and lstm_status returns the error with the CUDA
+ * context intact.  cta < 0 restores normal operation.  Nothing faults or hangs in either mode.
+ */
+LSTM_API int lstm_selftest_timeout(lstm_handle *h, int cta, long long spin_limit);
+
+/*
  * Measurement support.  With profiling on, lstm_forward brackets each of its kernels with CUDA events
  * on the launching stream; lstm_profile_read synchronises and returns, for the most recent
  * lstm_forward, per kernel kind k (LSTM_K_*): launches[k] and total device milliseconds ms[k].

@@ -64,6 +64,8 @@ def load_library():
         lib.lstm_profile_read.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ctypes.c_float)]
         lib.lstm_info.restype = ci
         lib.lstm_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), ci]
+        lib.lstm_selftest_timeout.restype = ci
+        lib.lstm_selftest_timeout.argtypes = [vp, ci, ctypes.c_longlong]
         lib.lstm_forward_noalloc.restype = ci
         lib.lstm_forward_noalloc.argtypes = [vp, vp, vp, ci, ci, vp, ci, ci, vp, vp, vp, vp, vp, vp, ctypes.c_char_p, ci]
         _lib = lib
@@ -100,6 +102,10 @@ def lstm_status(handle):
 
 def lstm_destroy(handle):
     return load_library().lstm_destroy(handle)
+
+
+def lstm_selftest_timeout(handle, cta, spin_limit=0):
+    return load_library().lstm_selftest_timeout(handle, cta, spin_limit)
 
 
 def lstm_profile_enable(handle, on):
@@ -251,6 +257,9 @@ class LSTM:
 
     def info(self):
         return lstm_info(self._handle)
+
+    def selftest_timeout(self, cta, spin_limit=0):
+        self._check(lstm_selftest_timeout(self._handle, cta, spin_limit))
 
     def profile_enable(self, on=True):
         self._check(lstm_profile_enable(self._handle, on))

@@ -57,6 +57,8 @@ struct lstm_handle {
     int *status_dev = nullptr;
     unsigned stamp_next = 0;
     long long spin_limit = 2000000000LL;
+    long long spin_limit_default = 2000000000LL;
+    int withhold_cta = -1;             // failure-path self-test (lstm_selftest_timeout)
     cudaStream_t last_stream = nullptr;
     // host-buffer variant staging
     float *hx = nullptr, *hy = nullptr, *hh0 = nullptr, *hc0 = nullptr, *hhT = nullptr, *hcT = nullptr;
@@ -388,6 +390,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     plan_mma(h);
     h->layers.resize(layers);
     if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
+    h->spin_limit_default = h->spin_limit;
 
     int rc = LSTM_OK;
     auto bail = [&](int code) { g_create_error = h->err; free_all(h); delete h; return code; };
@@ -667,6 +670,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.stamp_base = h->stamp_next;
             h->stamp_next += (unsigned)T + 1u;
             m.spin_limit = h->spin_limit;
+            m.withhold_cta = h->withhold_cta;
             for (int d = 0; d < D; ++d) m.wfrag[d] = ly.wfrag[d];
             m.G = h->G;
             m.g_split_stride = (long long)M * N;
@@ -693,6 +697,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         a.stamp_base = h->stamp_next;
         h->stamp_next += (unsigned)T + 1u;
         a.spin_limit = h->spin_limit;
+        a.withhold_cta = h->withhold_cta;
         for (int d = 0; d < D; ++d) { a.wh[d] = ly.wh[d]; a.csr_ptr[d] = ly.wh_ptr[d]; a.csr_ent[d] = ly.wh_ent[d]; }
         a.G = h->G;
         a.g_split_stride = (long long)M * N;
@@ -770,6 +775,15 @@ int lstm_destroy(lstm_handle *h)
     cudaDeviceSynchronize();
     free_all(h);
     delete h;
+    return LSTM_OK;
+}
+
+int lstm_selftest_timeout(lstm_handle *h, int cta, long long spin_limit)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    if (cta >= h->ncta_dir * h->D) return fail(h, LSTM_ERR_INVALID, "cta %d outside the launch of %d CTAs", cta, h->ncta_dir * h->D);
+    h->withhold_cta = cta < 0 ? -1 : cta;
+    h->spin_limit = spin_limit > 0 ? spin_limit : h->spin_limit_default;
     return LSTM_OK;
 }
 

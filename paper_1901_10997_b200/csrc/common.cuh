@@ -26,6 +26,7 @@ struct RecurArgs {
     int w_smem_bytes;   // shared-memory bytes set aside for resident weights
     unsigned stamp_base;        // exchange words of step s carry stamp_base + s + 1
     long long spin_limit;       // clock64 ticks a wait may last before the kernel gives up
+    int withhold_cta;           // failure-path self-test: this CTA never publishes its h values (-1: none)
     // dense: [H][4][Hp8] (unit-major, gates i,f,g,o); element type = weight type
     const void *wh[2];
     // CSR: per direction, rows in the same unit-major order; entry_ptr[4H+1] counts entries padded
@@ -64,6 +65,7 @@ struct RecurMmaArgs {
     int nkw_smem;               // trailing column tiles of every warp kept in shared memory
     unsigned stamp_base;
     long long spin_limit;
+    int withhold_cta;           // failure-path self-test: this CTA never publishes its h values (-1: none)
     // per direction [cta][warp][column tile][row tile][lane] 16-byte operand-A fragments:
     // lane (g = lane / 4, p = lane % 4) holds rows g and g + 8, columns 2p, 2p+1 and 2p+8, 2p+9
     const uint4 *wfrag[2];

@@ -377,6 +377,7 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
                     const AT cn_a = fma(vf, (AT)c_s[u * B + b], vi * vg);
                     const float cn = (float)cn_a;
                     const float hn = (float)(vo * tanh_t(cn_a));
+                    if ((int)blockIdx.x != a.withhold_cta)
                     st_relaxed_u64(xch_d + ((size_t)(s & 1) * B + b) * H + j,
                                    ((unsigned long long)(a.stamp_base + (unsigned)s + 1u) << 32) |
                                        (unsigned long long)__float_as_uint(hn));

@@ -295,6 +295,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                     const int b = b0 + fb, j = u0 + warp;
                     const float cn = fmaf(vf, c_s[warp * B + b], vi * vg);
                     const float hn = vo * tanh_fast(cn);
+                    if ((int)blockIdx.x != a.withhold_cta)
                     st_relaxed_u64(xch_d + ((size_t)(s & 1) * B + b) * H + j,
                                    ((unsigned long long)(a.stamp_base + (unsigned)s + 1u) << 32) |
                                        (unsigned long long)__float_as_uint(hn));

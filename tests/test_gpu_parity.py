@@ -180,3 +180,46 @@ def test_config5_b16_sampled_columns(oracle):
     for b in (3, 15):
         ref = oracle.forward(weights, x[:, b:b + 1], layers=w.layers, bidir=w.bidir, hidden=w.hidden)
         assert_close((y[:, b:b + 1], hT[:, b:b + 1], cT[:, b:b + 1]), ref, w.dtype, f"{w.name} col {b}")
+
+
+# ---------------------------------------------------------------- kernel selection and the failure path
+def test_shared_memory_kernel_serves_bf16_dense_when_selected(oracle, monkeypatch):
+    """bf16 dense weights normally run on the register-resident kernel; the shared-memory kernel is its
+    fall-back for slices that do not fit and must stay correct."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = small("simt_bf16", 2, True, 64, 149, 6, 3, "bf16", seed=21)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    for env, resident in (("simt", 0), ("", 1)):
+        monkeypatch.setenv("LSTM_B200_RECUR", env)
+        m = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=True, dtype="bf16",
+                     max_T=w.T, max_B=w.B)
+        assert m.info()["recur_register_resident"] == resident
+        y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
+        m.check()
+        assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"recur={env or 'default'}")
+        m.close()
+
+
+@pytest.mark.parametrize("dtype,mode", [("bf16", "dense"), ("fp32", "dense"), ("bf16", "csr")])
+def test_withheld_exchange_words_end_in_a_timeout_status_not_a_hang(oracle, dtype, mode):
+    """One CTA withholds its h values; the waits of the others run out after a millisecond, the call
+    reports LSTM_ERR_TIMEOUT, and the same handle computes correctly again afterwards."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = small("timeout", 1, False, 40, 300, 8, 2, dtype, seed=22)
+    weights, x = wl.make(w)
+    ref = oracle.forward(weights, x, layers=1, bidir=False, hidden=w.hidden)
+    m = pkg.LSTM(weights, layers=1, in_dim=w.in_dim, hidden=w.hidden, dtype=dtype, exec_mode=mode, max_T=w.T, max_B=w.B)
+    xd = torch.from_numpy(x).cuda()
+    m.selftest_timeout(5, 2_000_000)              # about a millisecond of clock ticks
+    m.forward(xd)
+    assert m.status() == pkg.LSTM_ERR_TIMEOUT
+    assert "timeout" in pkg.lstm_last_error(m.handle)
+    m.selftest_timeout(-1)
+    y, hT, cT = m.forward(xd)
+    m.check()
+    assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, dtype, "after the timeout")
+    m.close()
