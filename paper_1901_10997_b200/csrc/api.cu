@@ -234,14 +234,19 @@ void unit_range_host(int H, int nc, int c, int &u0, int &n)
 }
 
 // Launch shape of the recurrent kernel for B batch rows.
-struct RecurShape { int BT; size_t smem; int w_smem_bytes; int units_res_min; };
+struct RecurShape { int BT; size_t smem; int w_smem_bytes; int units_res_min; bool staged = false; };
 
 RecurShape recur_shape(const lstm_handle *h, int B, int layer)
 {
     if (h->use_mma) {
         RecurShape s;
         s.BT = 4;
-        s.smem = recur_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc, B);
+        // several batch rows: the exchange words land in shared memory (16-byte copies need an even H,
+        // at most 12 pairs per lane, and room for the landing area)
+        const int kspan = (h->mma_nkr + h->mma_nks) * 16;
+        s.staged = B > 1 && (h->H % 2) == 0 && 4 * kspan <= 64 * 12 &&
+                   recur_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc, B, true) <= (size_t)h->smem_optin - 64;
+        s.smem = recur_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc, B, s.staged);
         s.w_smem_bytes = h->mma_nw * h->mma_nks * h->mma_mt * 512;
         s.units_res_min = 0;
         return s;
@@ -303,7 +308,7 @@ void plan_mma(lstm_handle *h)
     if (nkr == 0) return;
     const int nks = need > nkr ? need - nkr : 0;
     if (!recur_mma_shape_ok(mt, nkr, nw)) return;
-    if (recur_mma_smem_bytes(mt, nkr, nw, nks, h->upc, h->max_B) > (size_t)h->smem_optin - 64) return;
+    if (recur_mma_smem_bytes(mt, nkr, nw, nks, h->upc, h->max_B, false) > (size_t)h->smem_optin - 64) return;
     h->use_mma = true;
     h->mma_mt = mt; h->mma_nkr = nkr; h->mma_nks = nks; h->mma_nw = nw;
 }
@@ -666,7 +671,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (h->use_mma) {
             RecurMmaArgs m;
             memset(&m, 0, sizeof m);
-            m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit; m.nkw_smem = h->mma_nks;
+            m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit; m.nkw_smem = h->mma_nks; m.staged = shp.staged ? 1 : 0;
             m.stamp_base = h->stamp_next;
             h->stamp_next += (unsigned)T + 1u;
             m.spin_limit = h->spin_limit;

@@ -63,6 +63,7 @@ struct RecurMmaArgs {
     int ncta_dir;
     int nsplit;
     int nkw_smem;               // trailing column tiles of every warp kept in shared memory
+    int staged;                 // 1: passes over several batch rows land their exchange words in shared memory
     unsigned stamp_base;
     long long spin_limit;
     int withhold_cta;           // failure-path self-test: this CTA never publishes its h values (-1: none)
@@ -83,7 +84,7 @@ struct RecurMmaArgs {
 constexpr int kMmaTileCap16 = 18;   // MT * NKR limit with 16 warps (128 registers per thread, no spills)
 constexpr int kMmaTileCap8 = 40;    // ... with 8 warps
 bool recur_mma_shape_ok(int mt, int nkr, int nw);
-size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B);
+size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B, bool staged);
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 

@@ -54,6 +54,15 @@ __device__ __forceinline__ float ld_nc_early(const float *p)
     asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
     return v;
 }
+// 16-byte asynchronous copy global -> shared through L2 only (never a stale L1 line)
+__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
 __device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ void bar_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
@@ -83,6 +92,7 @@ __device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n
 
 constexpr int kPoll = 4;      // exchange words a lane keeps in flight per polling round
 constexpr int kMaxSplit = 4;  // split-K planes of the projection output (the projection plans at most 4)
+constexpr int kMaxPairs = 12;  // pairs of exchange words per lane in a staged pass: 4 rows x up to 192 columns
 constexpr int kChunk = 4;     // batch rows per pass: hi and lo parts fill the 8 columns of the B operand
 
 // MT: 16-row tiles per CTA (4 gate rows x units, padded); NKR: 16-column tiles per warp held in
@@ -112,6 +122,8 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
     float *red = reinterpret_cast<float *>(smem + (size_t)NW * nkw * 256);        // [2][NW][WS] as [4][RP] + pad
     float *c_s = red + 2 * NW * WS;                                           // [upc][B]
     uint4 *As = reinterpret_cast<uint4 *>(c_s + ((upc * B + 3) & ~3));            // [NW][nks][MT][32]
+    // landing area of the exchange words of a pass over several batch rows: [NW][kChunk][kspan]
+    unsigned long long *stage = reinterpret_cast<unsigned long long *>(As + (size_t)NW * nks * MT * 32);
 
     // ---- residency: this warp's tiles, registers first, the rest in shared memory
     const uint4 *wsrc = a.wfrag[d] + ((size_t)(cta * NW + warp) * nkw) * MT * 32 + lane;
@@ -202,6 +214,62 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                         const __nv_bfloat16 hi = __float2bfloat16_rn(v);
                         Bw[dof] = hi;
                         Bw[dof + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
+                    }
+                }
+            } else if (a.staged) {
+                // Several batch rows: too many words per lane to hold in registers at once, and polling
+                // them in rounds would cost one L2 round trip per round.  All words of the pass are
+                // copied to shared memory asynchronously in one go (pairs of words, 16 bytes); pairs whose
+                // stamps are not there yet are requested again.
+                const unsigned want = a.stamp_base + (unsigned)s;
+                const unsigned long long *src = xch_d + ((size_t)((s - 1) & 1) * B + b0) * H + kbase;
+                unsigned long long *stg = stage + (size_t)warp * kChunk * kspan;
+                unsigned todo = 0;                                     // bit j: pair 2*lane + 64*j still missing
+#pragma unroll
+                for (int j = 0; j < kMaxPairs; ++j) {
+                    const int idx = 2 * lane + 64 * j;
+                    if (idx < nwords) {
+                        const int b = (idx >= kspan) + (idx >= 2 * kspan) + (idx >= 3 * kspan), kk = idx - b * kspan;
+                        if (kbase + kk < H) todo |= 1u << j;
+                    }
+                }
+                if (*abort_v) todo = 0;
+                long long t_start = 0;
+                int rounds = 0;
+                while (__any_sync(0xffffffffu, todo != 0)) {
+#pragma unroll
+                    for (int j = 0; j < kMaxPairs; ++j)
+                        if (todo & (1u << j)) {
+                            const int idx = 2 * lane + 64 * j;
+                            const int b = (idx >= kspan) + (idx >= 2 * kspan) + (idx >= 3 * kspan), kk = idx - b * kspan;
+                            cp_async_16(stg + idx, src + (size_t)b * H + kk);
+                        }
+                    cp_async_wait_all();
+#pragma unroll
+                    for (int j = 0; j < kMaxPairs; ++j)
+                        if (todo & (1u << j)) {
+                            const int idx = 2 * lane + 64 * j;
+                            const ulonglong2 w = *reinterpret_cast<const ulonglong2 *>(stg + idx);
+                            if ((unsigned)(w.x >> 32) == want && (unsigned)(w.y >> 32) == want) {
+                                const int b = (idx >= kspan) + (idx >= 2 * kspan) + (idx >= 3 * kspan), kk = idx - b * kspan;
+                                const float v0 = __uint_as_float((unsigned)w.x), v1 = __uint_as_float((unsigned)w.y);
+                                const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
+                                const __nv_bfloat162 lo = __floats2bfloat162_rn(v0 - __low2float(hi), v1 - __high2float(hi));
+                                const int dof = ((kk >> 4) * 8 + 2 * b) * 16 + (kk & 15);      // kk even: one 32-bit store
+                                *reinterpret_cast<__nv_bfloat162 *>(Bw + dof) = hi;
+                                *reinterpret_cast<__nv_bfloat162 *>(Bw + dof + 16) = lo;
+                                todo &= ~(1u << j);
+                            }
+                        }
+                    if (todo && ((++rounds & 15) == 0)) {
+                        const long long now = clock64();
+                        if (t_start == 0) t_start = now;
+                        if (*abort_v) todo = 0;
+                        else if (now - t_start > a.spin_limit || ld_volatile_s32(a.status) != kStatusOk) {
+                            *abort_v = 1;
+                            atomicExch(a.status, kStatusTimeout);
+                            todo = 0;
+                        }
                     }
                 }
             } else {
@@ -363,10 +431,10 @@ bool recur_mma_shape_ok(int mt, int nkr, int nw)
     return false;
 }
 
-size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B)
+size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B, bool staged)
 {
     const int nkw = nkr + nkw_smem;
-    return (size_t)nw * nkw * 256 + (size_t)2 * nw * (4 * (mt * 16 + 8) + 4) * 4 + (size_t)((upc * B + 3) & ~3) * 4 +
+    return (staged ? (size_t)nw * kChunk * nkw * 16 * 8 : 0) + (size_t)nw * nkw * 256 + (size_t)2 * nw * (4 * (mt * 16 + 8) + 4) * 4 + (size_t)((upc * B + 3) & ~3) * 4 +
            (size_t)nw * nkw_smem * mt * 512;
 }
 
