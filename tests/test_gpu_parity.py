@@ -8,8 +8,8 @@ from gpu_util import assert_close, csr_weights, run_gpu
 pytestmark = pytest.mark.gpu
 
 
-def small(name, L, bidir, in_dim, H, T, B, dtype, density=1.0, seed=1):
-    return wl.Workload(name, L, bidir, in_dim, H, T, B, dtype, 0.3, density=density, seed=seed)
+def small(name, L, bidir, in_dim, H, T, B, dtype, density=1.0, seed=1, scale=0.3):
+    return wl.Workload(name, L, bidir, in_dim, H, T, B, dtype, scale, density=density, seed=seed)
 
 
 # awkward shapes: H not a multiple of 8/32/148, H = 1, T = 1, B not a power of two, in != H
@@ -24,6 +24,10 @@ SHAPES = [
     small("h300_b16", 1, False, 96, 300, 5, 16, "fp32"),
     small("h200_b20", 3, True, 50, 200, 4, 20, "bf16"),
     small("h513_b9", 1, False, 130, 513, 3, 9, "bf16"),
+    # register-resident kernel with part of the slice in shared memory, several batch rows (register polling)
+    small("h1896_b3", 1, False, 72, 1896, 3, 3, "bf16", scale=0.03),      # weights ~ 1/sqrt(H) as in the sweep
+    # two passes of four rows with the staged exchange, both directions
+    small("h640_b7", 1, True, 48, 640, 4, 7, "bf16"),
 ]
 
 
