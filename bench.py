@@ -339,7 +339,7 @@ def run_gpu(args):
         line = {
             "metric": "us_per_sequence", "value": us_per_seq, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32",
+            "vs_baseline": None, "dtype": ("bf16" if w.dtype == "bf16" else "f32"),
             "data": "synthetic",
             "config": {"workload": w.name, "layers": w.layers, "dirs": w.dirs, "in_dim": w.in_dim, "hidden": w.hidden,
                        "T": w.T, "B": w.B, "exec_mode": mode, "weights": w.dtype, "state": "fp32", "l2": "flushed between timed steps (256 MiB write)",

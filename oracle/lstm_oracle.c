@@ -163,6 +163,119 @@ int lstm_oracle_forward(int L, int D, int in_dim, int H, int T, int B, const ora
     return rc;
 }
 
+/*
+ * H-LSTM variant (paper, Section 4, same equation block with H* = ONE hidden layer inside each gate:
+ * "hidden layer that performs a linear transformation followed by an activation function", here ReLU,
+ * one of the internal activations the paper names).  For gate q in {i,f,g,o}, hidden width Hh:
+ *
+ *     r_q = relu(a_q + Ux_q x_t + Uh_q h_{t-1})                (Hh values; U_q = [Ux_q | Uh_q] acts on [x_t, h_{t-1}])
+ *     z_q = b_q + W_q r_q                                       (H values)
+ *     i = sigma(z_i)  f = sigma(z_f)  g = tanh(z_g)  o = sigma(z_o)   c_t = f c_{t-1} + i g   h_t = o tanh(c_t)
+ *
+ * Layout: ux [4Hh, in_l] and uh [4Hh, H] with row q*Hh + m; a [4Hh]; w [4H, Hh] with row q*H + j (block q
+ * multiplies r_q); b [4H]; NULL biases are zeros.  Stacking, directions and state indexing as above.
+ */
+typedef struct {
+    const float *ux, *uh, *a, *w, *b;
+} oracle_hweights;
+
+static int run_direction_h(int in_l, int H, int Hh, int T, int B, int reverse, const oracle_hweights *w,
+                           const double *X, const double *h0, const double *c0,
+                           double *Y, int y_stride, int y_off, double *hT, double *cT)
+{
+    size_t n = (size_t)B * H, nr = (size_t)B * 4 * Hh;
+    double *h_prev = (double *)calloc(n ? n : 1, sizeof(double));
+    double *c_prev = (double *)calloc(n ? n : 1, sizeof(double));
+    double *h_new  = (double *)calloc(n ? n : 1, sizeof(double));
+    double *c_new  = (double *)calloc(n ? n : 1, sizeof(double));
+    double *r      = (double *)calloc(nr ? nr : 1, sizeof(double));
+    if (!h_prev || !c_prev || !h_new || !c_new || !r) { free(h_prev); free(c_prev); free(h_new); free(c_new); free(r); return 1; }
+    if (h0) memcpy(h_prev, h0, n * sizeof(double));
+    if (c0) memcpy(c_prev, c0, n * sizeof(double));
+
+    for (int s = 0; s < T; ++s) {
+        int t = reverse ? T - 1 - s : s;
+        /* hidden layers of the four gates */
+#ifdef _OPENMP
+#pragma omp parallel for collapse(2) schedule(static)
+#endif
+        for (int b = 0; b < B; ++b) {
+            for (int m = 0; m < 4 * Hh; ++m) {
+                const double *x_t = X + ((size_t)t * B + b) * in_l;
+                const double *h_p = h_prev + (size_t)b * H;
+                double acc = w->a ? (double)w->a[m] : 0.0;
+                for (int k = 0; k < in_l; ++k) acc += (double)w->ux[(size_t)m * in_l + k] * x_t[k];
+                for (int k = 0; k < H; ++k) acc += (double)w->uh[(size_t)m * H + k] * h_p[k];
+                r[(size_t)b * 4 * Hh + m] = acc > 0.0 ? acc : 0.0;
+            }
+        }
+        /* gate pre-activations from the hidden layers, gates, state update */
+#ifdef _OPENMP
+#pragma omp parallel for collapse(2) schedule(static)
+#endif
+        for (int b = 0; b < B; ++b) {
+            for (int j = 0; j < H; ++j) {
+                double z[4];
+                for (int q = 0; q < 4; ++q) {
+                    int row = q * H + j;
+                    const double *rq = r + (size_t)b * 4 * Hh + (size_t)q * Hh;
+                    double acc = w->b ? (double)w->b[row] : 0.0;
+                    for (int m = 0; m < Hh; ++m) acc += (double)w->w[(size_t)row * Hh + m] * rq[m];
+                    z[q] = acc;
+                }
+                double gi = sigma(z[0]);
+                double gf = sigma(z[1]);
+                double gg = tanh(z[2]);
+                double go = sigma(z[3]);
+                double c = gf * c_prev[(size_t)b * H + j] + gi * gg;
+                double h = go * tanh(c);
+                c_new[(size_t)b * H + j] = c;
+                h_new[(size_t)b * H + j] = h;
+                Y[((size_t)t * B + b) * y_stride + y_off + j] = h;
+            }
+        }
+        double *tmp;
+        tmp = h_prev; h_prev = h_new; h_new = tmp;
+        tmp = c_prev; c_prev = c_new; c_new = tmp;
+    }
+    if (hT) memcpy(hT, h_prev, n * sizeof(double));
+    if (cT) memcpy(cT, c_prev, n * sizeof(double));
+    free(h_prev); free(c_prev); free(h_new); free(c_new); free(r);
+    return 0;
+}
+
+int hlstm_oracle_forward(int L, int D, int in_dim, int H, int Hh, int T, int B, const oracle_hweights *w,
+                         const double *x, const double *h0, const double *c0,
+                         double *y, double *hT, double *cT)
+{
+    if (L < 1 || (D != 1 && D != 2) || in_dim < 1 || H < 1 || Hh < 1 || T < 0 || B < 0 || !w || !y) return 1;
+    if (T > 0 && B > 0 && !x) return 1;
+    for (int i = 0; i < L * D; ++i) if (!w[i].ux || !w[i].uh || !w[i].w) return 1;
+    size_t out_n = (size_t)T * B * D * H;
+    size_t st_n = (size_t)B * H;
+    double *cur = NULL, *nxt = NULL;
+    if (L > 1) {
+        cur = (double *)malloc((out_n ? out_n : 1) * sizeof(double));
+        nxt = (double *)malloc((out_n ? out_n : 1) * sizeof(double));
+        if (!cur || !nxt) { free(cur); free(nxt); return 1; }
+    }
+    const double *X = x;
+    int in_l = in_dim;
+    int rc = 0;
+    for (int l = 0; l < L && !rc; ++l) {
+        double *Y = (l == L - 1) ? y : nxt;
+        for (int d = 0; d < D && !rc; ++d) {
+            size_t s = (size_t)(l * D + d) * st_n;
+            rc = run_direction_h(in_l, H, Hh, T, B, d == 1, &w[l * D + d], X,
+                                 h0 ? h0 + s : NULL, c0 ? c0 + s : NULL,
+                                 Y, D * H, d * H, hT ? hT + s : NULL, cT ? cT + s : NULL);
+        }
+        if (l < L - 1) { double *tmp = cur; cur = nxt; nxt = tmp; X = cur; in_l = D * H; }
+    }
+    free(cur); free(nxt);
+    return rc;
+}
+
 int lstm_oracle_threads(void)
 {
 #ifdef _OPENMP

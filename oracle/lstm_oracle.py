@@ -47,9 +47,67 @@ def _load():
         lib = ctypes.CDLL(str(_LIB))
         lib.lstm_oracle_forward.restype = ctypes.c_int
         lib.lstm_oracle_forward.argtypes = [ctypes.c_int] * 6 + [ctypes.c_void_p] * 7
+        lib.hlstm_oracle_forward.restype = ctypes.c_int
+        lib.hlstm_oracle_forward.argtypes = [ctypes.c_int] * 7 + [ctypes.c_void_p] * 7
         lib.lstm_oracle_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
+
+
+class _HWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("ux", "uh", "a", "w", "b")]
+
+
+def forward_hlstm(weights, x, h0=None, c0=None, *, layers: int, bidir: bool, hidden: int, gate_hidden: int):
+    """H-LSTM stack (one ReLU hidden layer of width ``gate_hidden`` inside each gate; Section 4 with
+    H* = one layer).  Each (layer, direction) dict holds ``ux`` [4Hh,in_l], ``uh`` [4Hh,H], ``w`` [4H,Hh]
+    and optional ``a`` [4Hh], ``b`` [4H]; gate blocks i, f, g, o.  Returns (y, hT, cT) as float64."""
+    lib = _load()
+    L, D, H, Hh = int(layers), (2 if bidir else 1), int(hidden), int(gate_hidden)
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    T, B, in_dim = x.shape
+    if len(weights) != L * D:
+        raise ValueError("need one weight set per (layer, direction)")
+    keep = []
+
+    def f32(a, shape):
+        a = np.ascontiguousarray(a, dtype=np.float32)
+        if a.shape != shape:
+            raise ValueError(f"bad shape {a.shape}, expected {shape}")
+        keep.append(a)
+        return a
+
+    arr = (_HWeights * (L * D))()
+    for l in range(L):
+        in_l = in_dim if l == 0 else D * H
+        for d in range(D):
+            w, s = weights[l * D + d], arr[l * D + d]
+            s.ux = _ptr(f32(w["ux"], (4 * Hh, in_l)))
+            s.uh = _ptr(f32(w["uh"], (4 * Hh, H)))
+            s.w = _ptr(f32(w["w"], (4 * H, Hh)))
+            if w.get("a") is not None:
+                s.a = _ptr(f32(w["a"], (4 * Hh,)))
+            if w.get("b") is not None:
+                s.b = _ptr(f32(w["b"], (4 * H,)))
+
+    def state(a):
+        if a is None:
+            return None
+        a = np.ascontiguousarray(a, dtype=np.float64)
+        if a.shape != (L * D, B, H):
+            raise ValueError(f"bad state shape {a.shape}")
+        keep.append(a)
+        return a
+
+    h0, c0 = state(h0), state(c0)
+    y = np.zeros((T, B, D * H), dtype=np.float64)
+    hT = np.zeros((L * D, B, H), dtype=np.float64)
+    cT = np.zeros((L * D, B, H), dtype=np.float64)
+    rc = lib.hlstm_oracle_forward(L, D, in_dim, H, Hh, T, B, ctypes.cast(arr, ctypes.c_void_p),
+                                  _ptr(x), _ptr(h0), _ptr(c0), _ptr(y), _ptr(hT), _ptr(cT))
+    if rc != 0:
+        raise RuntimeError(f"hlstm_oracle_forward failed with code {rc}")
+    return y, hT, cT
 
 
 def threads() -> int:
