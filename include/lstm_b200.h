@@ -102,6 +102,30 @@ LSTM_API int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, 
                 const lstm_weights *w, int exec_mode, int max_T, int max_B, void *cuda_stream);
 
 /*
+ * H-LSTM cell (Section 4 with one hidden layer H inside each gate: a linear map followed by ReLU).  For
+ * gate q in {i,f,g,o}, hidden width Hh = gate_hidden:
+ *     r_q = relu(a_q + Ux_q x_t + Uh_q h_{t-1})        z_q = b_q + W_q r_q
+ * followed by the same gate functions and c/h update as above.  Weights of one (layer, direction), all
+ * row-major fp32, host or device pointers, read only during the call:
+ *   ux [4Hh, in_l], uh [4Hh, H]: rows q*Hh + m;  a [4Hh] or NULL;  w [4H, Hh]: row q*H + j multiplies r_q;
+ *   b [4H] or NULL.  A pruned weight is passed as an explicit zero (W (x) Msk).
+ * hlstm_create returns a handle that lstm_forward, lstm_forward_host, lstm_status, lstm_destroy and the
+ * other calls accept like an LSTM handle.  Only LSTM_BF16W_F32S storage is served; sizes whose per-CTA
+ * slices of Uh and W do not fit registers + shared memory (roughly hidden, gate_hidden > 1700) return
+ * LSTM_ERR_UNSUPPORTED.
+ */
+typedef struct {
+    const float *ux;
+    const float *uh;
+    const float *a;
+    const float *w;
+    const float *b;
+} hlstm_weights;
+
+LSTM_API int hlstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int gate_hidden, int bidir, int dtype,
+                 const hlstm_weights *w, int max_T, int max_B, void *cuda_stream);
+
+/*
  * Forward pass over a whole sequence batch; all pointers are DEVICE pointers owned by the caller.
  *   x  [T,B,in_dim]      h0, c0 [L*D,B,H] or NULL (zeros)
  *   y  [T,B,D*H]         hT, cT [L*D,B,H] or NULL (not wanted)

@@ -122,6 +122,28 @@ def make(w: Workload):
     return weights, x
 
 
+def make_hlstm(w: Workload, gate_hidden: int):
+    """Weights of the H-LSTM cell (one hidden layer of width ``gate_hidden`` inside each gate) with the
+    shape of workload ``w``: per (layer, direction) ``ux`` [4Hh,in_l], ``uh`` [4Hh,H], ``a`` [4Hh],
+    ``w`` [4H,Hh], ``b`` [4H], all ~ U(-scale, scale), rounded to the storage type; then ``x``."""
+    rng = np.random.Generator(np.random.PCG64(w.seed + 991))
+    store = round_to_bf16 if w.dtype == "bf16" else (lambda a: a)
+    H, Hh = w.hidden, gate_hidden
+    weights = []
+    for l in range(w.layers):
+        for _d in range(w.dirs):
+            in_l = w.in_l(l)
+            weights.append({
+                "ux": store(rng.uniform(-w.scale, w.scale, size=(4 * Hh, in_l)).astype(np.float32)),
+                "uh": store(rng.uniform(-w.scale, w.scale, size=(4 * Hh, H)).astype(np.float32)),
+                "a": store(rng.uniform(-w.scale, w.scale, size=(4 * Hh,)).astype(np.float32)),
+                "w": store(rng.uniform(-w.scale, w.scale, size=(4 * H, Hh)).astype(np.float32)),
+                "b": store(rng.uniform(-w.scale, w.scale, size=(4 * H,)).astype(np.float32)),
+            })
+    x = rng.standard_normal(size=(w.T, w.B, w.in_dim)).astype(np.float32)
+    return weights, x
+
+
 def make_states(w: Workload, seed_offset: int = 7):
     """Non-zero initial states h0 in (-1,1), c0 ~ N(0,0.5), float32 [L*D,B,H]."""
     rng = np.random.Generator(np.random.PCG64(w.seed + seed_offset))

@@ -4,7 +4,7 @@ Every step of the computation runs in the library's CUDA kernels; this package o
 arguments.  There is no CPU fallback: if the shared library is missing or no CUDA device is usable,
 the calls raise.
 """
-from .binding import (LSTM, LstmError, lib_path, load_library, lstm_create, lstm_destroy,  # noqa: F401
+from .binding import (LSTM, HLSTM, LstmError, hlstm_create, lib_path, load_library, lstm_create, lstm_destroy,  # noqa: F401
                       lstm_forward, lstm_forward_host, lstm_forward_noalloc, lstm_info, lstm_last_error,
                       lstm_profile_enable, lstm_profile_read, lstm_selftest_timeout, lstm_status,
                       LSTM_F32, LSTM_BF16W_F32S, LSTM_DENSE, LSTM_CSR, LSTM_OK, LSTM_ERR_INVALID,

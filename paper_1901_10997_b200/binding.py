@@ -32,6 +32,10 @@ class _Weights(ctypes.Structure):
                  "wh_rowptr", "wh_col", "wh_val")]
 
 
+class _HWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("ux", "uh", "a", "w", "b")]
+
+
 def lib_path() -> Path:
     return _LIB_PATH
 
@@ -48,6 +52,8 @@ def load_library():
         vp, ci = ctypes.c_void_p, ctypes.c_int
         lib.lstm_create.restype = ci
         lib.lstm_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, vp, ci, ci, ci, vp]
+        lib.hlstm_create.restype = ci
+        lib.hlstm_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, vp, ci, ci, vp]
         lib.lstm_forward.restype = ci
         lib.lstm_forward.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, vp, vp]
         lib.lstm_forward_host.restype = ci
@@ -83,6 +89,14 @@ def lstm_create(layers, in_dim, hidden, bidir, dtype, weights_ptr, exec_mode, ma
     out = ctypes.c_void_p()
     rc = load_library().lstm_create(ctypes.byref(out), layers, in_dim, hidden, int(bool(bidir)), dtype,
                                     weights_ptr, exec_mode, max_T, max_B, stream or None)
+    return rc, out.value
+
+
+def hlstm_create(layers, in_dim, hidden, gate_hidden, bidir, dtype, weights_ptr, max_T, max_B, stream=0):
+    """Returns (code, handle).  ``weights_ptr``: address of an hlstm_weights[layers*(1+bidir)] array."""
+    out = ctypes.c_void_p()
+    rc = load_library().hlstm_create(ctypes.byref(out), layers, in_dim, hidden, gate_hidden, int(bool(bidir)), dtype,
+                                     weights_ptr, max_T, max_B, stream or None)
     return rc, out.value
 
 
@@ -279,3 +293,34 @@ class LSTM:
             self.close()
         except Exception:
             pass
+
+
+class HLSTM(LSTM):
+    """H-LSTM cell (one ReLU hidden layer of width ``gate_hidden`` inside each gate).  ``weights``: list of
+    dicts per (layer, direction) with ``ux`` [4Hh,in_l], ``uh`` [4Hh,H], ``w`` [4H,Hh], optional ``a``, ``b``;
+    gate blocks i, f, g, o.  Forward, status and the other methods are those of ``LSTM``."""
+
+    def __init__(self, weights, *, layers, in_dim, hidden, gate_hidden, bidir=False, dtype="bf16", max_T, max_B, stream=0):
+        self.layers, self.in_dim, self.hidden = int(layers), int(in_dim), int(hidden)
+        self.gate_hidden = int(gate_hidden)
+        self.dirs = 2 if bidir else 1
+        self.max_T, self.max_B = int(max_T), int(max_B)
+        self._handle = None
+        n = self.layers * self.dirs
+        if len(weights) != n:
+            raise ValueError(f"need {n} weight sets, got {len(weights)}")
+        arr = (_HWeights * n)()
+        keep = []
+        for i, w in enumerate(weights):
+            s = arr[i]
+            s.ux = _addr(_as_c(w["ux"], np.float32), keep)
+            s.uh = _addr(_as_c(w["uh"], np.float32), keep)
+            s.w = _addr(_as_c(w["w"], np.float32), keep)
+            s.a = _addr(_as_c(w.get("a"), np.float32), keep)
+            s.b = _addr(_as_c(w.get("b"), np.float32), keep)
+        dt = {"fp32": LSTM_F32, "bf16": LSTM_BF16W_F32S}[dtype]
+        rc, handle = hlstm_create(self.layers, self.in_dim, self.hidden, self.gate_hidden, bidir, dt,
+                                  ctypes.cast(arr, ctypes.c_void_p), self.max_T, self.max_B, stream)
+        if rc != LSTM_OK:
+            raise LstmError(rc, lstm_last_error(None))
+        self._handle = handle

@@ -30,6 +30,8 @@ struct Layer {
     int *wh_ptr[2] = {nullptr, nullptr};   // CSR recurrence: padded entry offsets [4H+1]
     void *wh_ent[2] = {nullptr, nullptr};
     uint4 *wfrag[2] = {nullptr, nullptr};  // register-resident kernel: operand-A fragments
+    uint4 *frag2[2] = {nullptr, nullptr};  // H-LSTM: fragments of the gate output matrices W
+    float *bias_out = nullptr;             // H-LSTM: [D][H][4] bias of the gate pre-activations
     int csr_max_slice_entries = 0;     // largest per-CTA slice (entries, padded)
     ProjTcPlan plan;                   // tensor-core projection plan for plan_M rows
     int plan_M = -1;
@@ -47,6 +49,9 @@ struct lstm_handle {
     // in shared memory, warps per CTA
     bool use_mma = false;
     int mma_mt = 0, mma_nkr = 0, mma_nks = 0, mma_nw = 0;
+    // H-LSTM cell: width of the hidden layer inside each gate (0: plain LSTM), pass-2 column tiles per warp
+    int Hh = 0, hl_nkw2 = 0;
+    unsigned long long *rxch = nullptr; size_t rxch_words = 0;
     std::vector<Layer> layers;
     // workspace
     float *G = nullptr; size_t G_cap = 0;
@@ -327,10 +332,11 @@ void free_all(lstm_handle *h)
 {
     for (auto &ly : h->layers) {
         cudaFree(ly.wx); cudaFree(ly.bias); cudaFree(ly.wx_rowptr); cudaFree(ly.wx_ent);
-        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); }
+        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); cudaFree(ly.frag2[d]); }
+        cudaFree(ly.bias_out);
     }
     cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
-    cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->status_dev);
+    cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->rxch); cudaFree(h->status_dev);
     cudaFree(h->hx); cudaFree(h->hy); cudaFree(h->hh0); cudaFree(h->hc0); cudaFree(h->hhT); cudaFree(h->hcT);
     for (auto e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
@@ -574,6 +580,173 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     return LSTM_OK;
 }
 
+// Operand-A fragments of a [4U x K] matrix whose row q*U + u is gate q of unit u: per CTA (units split
+// evenly over ncta CTAs) [warp][column tile][row tile][lane] x 4 words, local row = 4 * unit + gate,
+// zero beyond the CTA's units and beyond column K.
+static std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int NW, int nkw, int MT)
+{
+    std::vector<uint32_t> f((size_t)ncta * NW * nkw * MT * 32 * 4, 0u);
+    size_t o = 0;
+    for (int c = 0; c < ncta; ++c) {
+        int u0, nu; unit_range_host(U, ncta, c, u0, nu);
+        auto wv = [&](int r, int k) -> uint32_t {
+            if (r >= 4 * nu || k >= K) return 0u;
+            return f32_to_bf16_rne(m[(size_t)((r & 3) * U + u0 + (r >> 2)) * K + k]);
+        };
+        for (int wp = 0; wp < NW; ++wp)
+            for (int i = 0; i < nkw; ++i)
+                for (int mt = 0; mt < MT; ++mt)
+                    for (int lane = 0; lane < 32; ++lane) {
+                        const int g = lane >> 2, p2 = (lane & 3) * 2;
+                        const int r0 = mt * 16 + g, r1 = r0 + 8;
+                        const int ka = (wp * nkw + i) * 16 + p2, kb = ka + 8;
+                        f[o++] = wv(r0, ka) | (wv(r0, ka + 1) << 16);
+                        f[o++] = wv(r1, ka) | (wv(r1, ka + 1) << 16);
+                        f[o++] = wv(r0, kb) | (wv(r0, kb + 1) << 16);
+                        f[o++] = wv(r1, kb) | (wv(r1, kb + 1) << 16);
+                    }
+    }
+    return f;
+}
+
+int hlstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int gate_hidden, int bidir, int dtype,
+                 const hlstm_weights *w, int max_T, int max_B, void *cuda_stream)
+{
+    if (!out) return fail(nullptr, LSTM_ERR_INVALID, "out is NULL");
+    *out = nullptr;
+    if (layers < 1 || in_dim < 1 || hidden < 1 || gate_hidden < 1 || (bidir != 0 && bidir != 1) || !w || max_T < 1 || max_B < 1)
+        return fail(nullptr, LSTM_ERR_INVALID, "bad argument: layers=%d in_dim=%d hidden=%d gate_hidden=%d bidir=%d max_T=%d max_B=%d w=%p",
+                    layers, in_dim, hidden, gate_hidden, bidir, max_T, max_B, (const void *)w);
+    if (dtype != LSTM_F32 && dtype != LSTM_BF16W_F32S) return fail(nullptr, LSTM_ERR_INVALID, "unknown dtype %d", dtype);
+    if (dtype != LSTM_BF16W_F32S) return fail(nullptr, LSTM_ERR_UNSUPPORTED, "the H-LSTM cell is served with bf16 weights only");
+    if (hidden >= 65536 || gate_hidden >= 65536) return fail(nullptr, LSTM_ERR_UNSUPPORTED, "hidden widths must be < 65536");
+    if ((long long)max_T * max_B > (1LL << 30)) return fail(nullptr, LSTM_ERR_UNSUPPORTED, "max_T*max_B too large");
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        const char *m = cudaGetErrorString(cudaGetLastError());
+        return fail(nullptr, LSTM_ERR_CUDA, "no usable CUDA device: %s", m);
+    }
+    if (prop.major != 10) return fail(nullptr, LSTM_ERR_CUDA, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+    int coop = 0;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (!coop) return fail(nullptr, LSTM_ERR_CUDA, "device does not support cooperative launch");
+
+    lstm_handle *h = new (std::nothrow) lstm_handle;
+    if (!h) return fail(nullptr, LSTM_ERR_NOMEM, "host allocation failed");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int H = hidden, Hh = gate_hidden, D = bidir ? 2 : 1;
+    h->L = layers; h->D = D; h->in_dim = in_dim; h->H = H; h->Hh = Hh; h->dtype = dtype;
+    h->exec_mode = LSTM_DENSE; h->max_T = max_T; h->max_B = max_B; h->device = dev;
+    h->sm_count = prop.multiProcessorCount;
+    h->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    h->last_stream = st;
+    h->Hp8 = round_up(H, 8); h->Hs = round_up(H, 256);
+    h->ncta_dir = std::max(1, std::min(h->sm_count / D, std::min(H, Hh)));
+    h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
+    h->threads = 512;
+    h->use_tc = true;
+    h->layers.resize(layers);
+    if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
+    h->spin_limit_default = h->spin_limit;
+    auto bail = [&](int code) { g_create_error = h->err; free_all(h); delete h; return code; };
+
+    // tiling: row tiles cover 4 x (units per CTA) of both passes; pass 1 keeps up to nkr column tiles per
+    // warp in registers, the rest and all of pass 2 in shared memory
+    {
+        const int upch = (Hh + h->ncta_dir - 1) / h->ncta_dir;
+        const int mt = (4 * std::max(h->upc, upch) + 15) / 16;
+        const int nk1 = (H + 15) / 16, nk2 = (Hh + 15) / 16;
+        const int nw = (nk1 <= 32 && nk2 <= 32 && std::max(h->upc, upch) <= 8) ? 8 : 16;
+        const int need1 = (nk1 + nw - 1) / nw, need2 = (nk2 + nw - 1) / nw;
+        bool ok = mt <= 4 && std::max(h->upc, upch) <= nw;
+        int nkr = 0;
+        if (ok) {
+            const int cap = (nw == 16 ? kMmaTileCap16 : kMmaTileCap8) / mt;
+            for (int c = 2; c <= 8; c += 2)
+                if (c <= cap && (nkr == 0 || nkr < need1)) nkr = c;
+            ok = nkr > 0 && recur_mma_shape_ok(mt, nkr, nw);
+        }
+        const int nks1 = ok && need1 > nkr ? need1 - nkr : 0;
+        if (ok) ok = hlstm_mma_smem_bytes(mt, nkr, nw, nks1, need2, h->upc, max_B) <= (size_t)h->smem_optin - 64;
+        if (!ok) {
+            fail(h, LSTM_ERR_UNSUPPORTED, "hidden=%d gate_hidden=%d max_B=%d: the per-CTA slices do not fit registers and shared memory", H, Hh, max_B);
+            return bail(LSTM_ERR_UNSUPPORTED);
+        }
+        h->use_mma = true;
+        h->mma_mt = mt; h->mma_nkr = nkr; h->mma_nks = nks1; h->mma_nw = nw; h->hl_nkw2 = need2;
+    }
+
+    int rc = LSTM_OK;
+    for (int l = 0; l < layers && rc == LSTM_OK; ++l) {
+        Layer &ly = h->layers[l];
+        ly.in_l = l == 0 ? in_dim : D * H;
+        ly.ldk = round_up(ly.in_l, 8);
+        const int N = D * 4 * Hh;
+        std::vector<float> bias_p((size_t)N, 0.0f), bias_o((size_t)D * 4 * H, 0.0f);
+        std::vector<uint16_t> wx16((size_t)N * ly.ldk, 0);
+        for (int d = 0; d < D && rc == LSTM_OK; ++d) {
+            const hlstm_weights &src = w[l * D + d];
+            if (!src.ux || !src.uh || !src.w) { rc = fail(h, LSTM_ERR_INVALID, "ux, uh and w must be given (layer %d, dir %d)", l, d); break; }
+            HostView v_ux, v_uh, v_w, v_a, v_b;
+            if (!host_view(src.ux, sizeof(float) * 4 * Hh * ly.in_l, v_ux) || !host_view(src.uh, sizeof(float) * 4 * Hh * H, v_uh) ||
+                !host_view(src.w, sizeof(float) * 4 * H * Hh, v_w) || !host_view(src.a, sizeof(float) * 4 * Hh, v_a) ||
+                !host_view(src.b, sizeof(float) * 4 * H, v_b)) { rc = fail(h, LSTM_ERR_CUDA, "reading weights"); break; }
+            const float *ux = (const float *)v_ux.ptr, *uh = (const float *)v_uh.ptr, *ww = (const float *)v_w.ptr;
+            const float *ba = (const float *)v_a.ptr, *bb = (const float *)v_b.ptr;
+            for (int q = 0; q < 4; ++q) {
+                for (int m = 0; m < Hh; ++m) {
+                    const size_t prow = (size_t)d * 4 * Hh + (size_t)m * 4 + q;           // unit-major, gates adjacent
+                    if (ba) bias_p[prow] = ba[q * Hh + m];
+                    const float *srow = ux + (size_t)(q * Hh + m) * ly.in_l;
+                    for (int k = 0; k < ly.in_l; ++k) wx16[prow * ly.ldk + k] = f32_to_bf16_rne(srow[k]);
+                }
+                if (bb) for (int j = 0; j < H; ++j) bias_o[(size_t)d * 4 * H + (size_t)j * 4 + q] = bb[q * H + j];
+            }
+            const int NW = h->mma_nw;
+            std::vector<uint32_t> f1 = pack_fragments(uh, Hh, H, h->ncta_dir, NW, h->mma_nkr + h->mma_nks, h->mma_mt);
+            std::vector<uint32_t> f2 = pack_fragments(ww, H, Hh, h->ncta_dir, NW, h->hl_nkw2, h->mma_mt);
+            rc = upload(h, (uint32_t **)&ly.wfrag[d], f1.data(), f1.size() * 4, st, "hidden-layer recurrent fragments");
+            if (rc == LSTM_OK) rc = upload(h, (uint32_t **)&ly.frag2[d], f2.data(), f2.size() * 4, st, "gate output fragments");
+            if (rc == LSTM_OK) cudaStreamSynchronize(st);
+        }
+        if (rc) break;
+        rc = upload(h, &ly.bias, bias_p.data(), bias_p.size() * 4, st, "hidden-layer bias");
+        if (rc == LSTM_OK) rc = upload(h, &ly.bias_out, bias_o.data(), bias_o.size() * 4, st, "gate bias");
+        if (rc == LSTM_OK) rc = upload(h, (uint16_t **)&ly.wx, wx16.data(), wx16.size() * 2, st, "input weights");
+        if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)
+            rc = fail(h, LSTM_ERR_CUDA, "upload failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+    if (rc) return bail(rc);
+
+    const size_t Mmax = (size_t)max_T * max_B;
+    const size_t N = (size_t)D * 4 * Hh;
+    h->G_cap = std::max(Mmax * N, std::min<size_t>(Mmax, 256) * N * n_split_cap());
+    rc = dev_alloc(h, &h->G, h->G_cap * 4, false, st, "projection workspace");
+    h->ld0 = round_up(in_dim, 8);
+    if (rc == LSTM_OK) rc = dev_alloc(h, &h->xb0, 2 * Mmax * h->ld0 * 2, true, st, "bf16 input staging");
+    if (layers > 1) {
+        h->ldn = round_up(D * H, 8);
+        for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->xbn[i], 2 * Mmax * h->ldn * 2, true, st, "bf16 layer activations");
+        for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->ybuf[i], Mmax * D * H * 4, false, st, "layer activations");
+    }
+    h->xch_words = (size_t)D * 2 * max_B * H;
+    h->rxch_words = (size_t)D * 2 * max_B * 4 * Hh;
+    if (rc == LSTM_OK) rc = dev_alloc(h, &h->xch, h->xch_words * 8, true, st, "exchange buffer");
+    if (rc == LSTM_OK) rc = dev_alloc(h, &h->rxch, h->rxch_words * 8, true, st, "hidden-layer exchange buffer");
+    if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
+    if (rc == LSTM_OK) {
+        cudaError_t e = hlstm_mma_prepare(h->mma_mt, h->mma_nkr, h->mma_nw, h->smem_optin - 64);
+        if (e == cudaSuccess) e = proj_tc_prepare();
+        if (e != cudaSuccess) rc = fail(h, LSTM_ERR_CUDA, "kernel set-up failed: %s", cudaGetErrorString(e));
+    }
+    if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)
+        rc = fail(h, LSTM_ERR_CUDA, "workspace set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
+    if (rc) return bail(rc);
+    *out = h;
+    return LSTM_OK;
+}
+
 static int record(lstm_handle *h, int kind, cudaStream_t st)
 {
     if (!h->prof) return 0;
@@ -622,13 +795,14 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
     // stamps of the exchange words must stay unique: restart from a cleared buffer before wrapping
     if ((unsigned long long)h->stamp_next + (unsigned long long)L * T + 2ull >= 0xffffffffull) {
         if (cudaMemsetAsync(h->xch, 0, h->xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
+        if (h->rxch && cudaMemsetAsync(h->rxch, 0, h->rxch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         h->stamp_next = 0;
     }
 
     for (int l = 0; l < L; ++l) {
         Layer &ly = h->layers[l];
         const float *Xf = l == 0 ? x : h->ybuf[(l - 1) & 1];
-        const int N = D * 4 * H;
+        const int N = D * 4 * (h->Hh ? h->Hh : H);      // H-LSTM: the projection feeds the hidden layers
         int nsplit = 1;
         // ---- input staging + projection
         if (csr) {
@@ -667,6 +841,36 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "projection launch failed (layer %d): %s", l, cudaGetErrorString(e));
 
         // ---- recurrence
+        if (h->Hh) {
+            HlstmArgs m;
+            memset(&m, 0, sizeof m);
+            m.H = H; m.Hh = h->Hh; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
+            m.nks1 = h->mma_nks; m.nkw2 = h->hl_nkw2;
+            m.stamp_base = h->stamp_next;
+            h->stamp_next += (unsigned)T + 1u;
+            m.spin_limit = h->spin_limit;
+            m.withhold_cta = h->withhold_cta;
+            for (int d = 0; d < D; ++d) { m.frag1[d] = ly.wfrag[d]; m.frag2[d] = ly.frag2[d]; }
+            m.G = h->G;
+            m.g_split_stride = (long long)M * N;
+            m.bias_out = ly.bias_out;
+            const size_t so = (size_t)l * D * B * H;
+            m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
+            m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
+            m.y = l == L - 1 ? y : h->ybuf[l & 1];
+            m.xb_next = l < L - 1 ? h->xbn[l & 1] : nullptr;
+            m.xb_ld = h->ldn;
+            m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
+            m.xch = h->xch; m.rxch = h->rxch;
+            m.status = h->status_dev;
+            const size_t smem = hlstm_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->hl_nkw2, h->upc, B);
+            if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_hlstm_mma(m, h->mma_mt, h->mma_nkr, h->mma_nw, smem, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
+            continue;
+        }
         const RecurShape shp = recur_shape(h, B, l);
         if (h->use_mma) {
             RecurMmaArgs m;
@@ -821,7 +1025,8 @@ int lstm_profile_read(lstm_handle *h, int *launches, float *ms)
 int lstm_info(const lstm_handle *h, int64_t *out, int n)
 {
     if (!h || !out || n < 0) return 0;
-    const RecurShape shp = recur_shape(h, h->max_B, 0);
+    RecurShape shp = recur_shape(h, h->max_B, 0);
+    if (h->Hh) shp.smem = hlstm_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->hl_nkw2, h->upc, h->max_B);
     const size_t wsize = h->dtype == LSTM_BF16W_F32S ? 2 : 4;
     int64_t rows_res = 0, rows_str = 0;
     if (h->use_mma) {

@@ -89,6 +89,40 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------------
+// H-LSTM recurrent kernel (one ReLU hidden layer of width Hh inside each gate; bf16 weights, dense).
+// Pass 1 works on the four Uh_q [Hh x H] (hidden units split over the CTAs, fragments in registers and,
+// beyond nkr tiles per warp, in shared memory), pass 2 on the four W_q [H x Hh] (cell units split over the
+// CTAs, fragments in shared memory).  Fragment layout as in RecurMmaArgs.
+// ---------------------------------------------------------------------------------------------------
+struct HlstmArgs {
+    int H, Hh, B, T, D;
+    int ncta_dir;
+    int nsplit;
+    int nks1;                   // pass 1: column tiles per warp in shared memory (after the register tiles)
+    int nkw2;                   // pass 2: column tiles per warp (all in shared memory)
+    unsigned stamp_base;
+    long long spin_limit;
+    int withhold_cta;
+    const uint4 *frag1[2];      // Uh: local row = 4 * hidden unit + gate
+    const uint4 *frag2[2];      // W:  local row = 4 * cell unit + gate
+    const float *G;             // [nsplit][T*B][D][Hh][4] input half of the hidden layers incl. their bias
+    long long g_split_stride;
+    const float *bias_out;      // [D][H][4] bias of the gate pre-activations
+    const float *h0, *c0;
+    float *hT, *cT;
+    float *y;
+    __nv_bfloat16 *xb_next;
+    long long xb_plane;
+    int xb_ld;
+    unsigned long long *xch;    // [D][2][B][H] h words
+    unsigned long long *rxch;   // [D][2][B][4][Hh] hidden-layer words
+    int *status;
+};
+size_t hlstm_mma_smem_bytes(int mt, int nkr, int nw, int nks1, int nkw2, int upc, int B);
+cudaError_t hlstm_mma_prepare(int mt, int nkr, int nw, int max_smem);
+cudaError_t launch_hlstm_mma(const HlstmArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------
 // Input staging and projection
 // ---------------------------------------------------------------------------------------------------
 // x fp32 [M][K] -> two bf16 planes [M][ld]: hi = bf16(x), lo = bf16(x - hi) at xb + plane
