@@ -48,6 +48,10 @@ def pick_workload(name: str):
         "cfg4_05_csr": (wl.config4(0.05), "csr"),
         "cfg5": (wl.config5(1), "dense"),
         "cfg5_b16": (wl.config5(16), "dense"),
+        # H-LSTM cell (one ReLU hidden layer of the cell's width inside each gate), the paper's own models:
+        # one layer of width 1500 for the language model, three bidirectional layers of width 800 for speech
+        "hlstm_ptb": (wl.config2(1).with_(name="hlstm_ptb_1x1500_B1", layers=1), "hlstm"),
+        "hlstm_ds2": (wl.config5(1).with_(name="hlstm_ds2_3x2x800_B1", layers=3), "hlstm"),
     }
     return table[name]
 
@@ -81,6 +85,17 @@ def measured_traffic(kernel: str, workload: str, source: str):
     return int(m_tr.group(1))
 
 
+def make_inputs(w: wl.Workload, mode: str):
+    return wl.make_hlstm(w, w.hidden) if mode == "hlstm" else wl.make(w)
+
+
+def oracle_forward(w: wl.Workload, mode: str, weights, xs):
+    import oracle
+    if mode == "hlstm":
+        return oracle.forward_hlstm(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden, gate_hidden=w.hidden)
+    return oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+
+
 def recurrence_bytes_per_launch(w: wl.Workload, nnz_per_layer=None) -> float:
     """Algorithmic bytes one recurrent-kernel launch (one layer, all T steps, all directions) needs if
     nothing were resident: per step and direction the recurrent matrix once (4H*H*w bytes dense, or
@@ -88,7 +103,9 @@ def recurrence_bytes_per_launch(w: wl.Workload, nnz_per_layer=None) -> float:
     projection row read (B*4H*4)."""
     H, B, T, D = w.hidden, w.B, w.T, w.dirs
     wbytes = 2 if w.dtype == "bf16" else 4
-    if nnz_per_layer is None:
+    if nnz_per_layer == "hlstm":
+        mat = 2 * 4.0 * H * H * wbytes + B * 4.0 * H * 8.0      # Uh and W, plus the hidden-layer values exchanged
+    elif nnz_per_layer is None:
         mat = 4.0 * H * H * wbytes
     else:
         mat = nnz_per_layer / D * (wbytes + 2) + (4 * H + 1) * 4
@@ -147,18 +164,18 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def oracle_time(w: wl.Workload, weights, x, target_seconds=12.0, max_reps=50):
+def oracle_time(w: wl.Workload, weights, x, target_seconds=12.0, max_reps=50, mode="dense"):
     """Times the oracle as it stands on a bounded sample: whole sequences of the workload (for B > 1
     only the first batch column), repeated until ~target_seconds of wall time have passed."""
     import oracle
     xs = x[:, :1] if w.B > 1 else x
     t0 = time.perf_counter()
-    oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    oracle_forward(w, mode, weights, xs)
     first = time.perf_counter() - t0
     reps = int(max(1, min(max_reps, target_seconds / max(first, 1e-6))))
     t0 = time.perf_counter()
     for _ in range(reps):
-        oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        oracle_forward(w, mode, weights, xs)
     per_seq = (time.perf_counter() - t0) / reps
     return per_seq, reps, oracle.threads()
 
@@ -168,15 +185,15 @@ def run_reference(args):
     if rank != 0:
         return
     w, _mode = pick_workload(args.workload)
-    weights, x = wl.make(w)
+    weights, x = make_inputs(w, _mode)
     import oracle
     xs = x[:, :1] if w.B > 1 else x
     for _ in range(min(args.warmup, 1)):
-        oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        oracle_forward(w, _mode, weights, xs)
     steps = max(1, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle.forward(weights, xs, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        oracle_forward(w, _mode, weights, xs)
     per_seq = (time.perf_counter() - t0) / steps
     us = per_seq * 1e6
     sample = f"{steps} whole sequences of {w.name} (T={w.T}, one batch column per step), fp64 oracle"
@@ -238,11 +255,11 @@ def run_gpu(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     w, mode = pick_workload(args.workload)
-    weights, x = wl.make(w)
+    weights, x = make_inputs(w, mode)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        per_seq, reps, cores = oracle_time(w, weights, x)
+        per_seq, reps, cores = oracle_time(w, weights, x, mode=mode)
         cpu = {"value": per_seq * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
                "sample": f"{reps} whole sequences of {w.name} (T={w.T}, one batch column each) after one warm-up"}
 
@@ -255,8 +272,12 @@ def run_gpu(args):
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist = dist_mod
 
-    model = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
-                     exec_mode=mode, max_T=w.T, max_B=w.B)
+    if mode == "hlstm":
+        model = pkg.HLSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, gate_hidden=w.hidden, bidir=w.bidir,
+                          dtype=w.dtype, max_T=w.T, max_B=w.B)
+    else:
+        model = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
+                         exec_mode=mode, max_T=w.T, max_B=w.B)
     dev = torch.device("cuda", local_rank)
     xd = torch.from_numpy(x).to(dev)
     out = (torch.empty((w.T, w.B, w.dirs * w.hidden), device=dev),
@@ -329,11 +350,12 @@ def run_gpu(args):
         if mode == "csr":
             nnz = float(np.mean([sum(int(np.count_nonzero(weights[l * w.dirs + d]["mask_h"])) for d in range(w.dirs))
                                  for l in range(w.layers)]))
-        alg_bytes = recurrence_bytes_per_launch(w, nnz)
+        alg_bytes = recurrence_bytes_per_launch(w, "hlstm" if mode == "hlstm" else nnz)
         rec_avg_ms = rec_ms / max(rec_n, 1)
         achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
         info = model.info()
-        kernel_name, kernel_src = (("recur_mma_kernel", "recur_mma.cu") if info.get("recur_register_resident")
+        kernel_name, kernel_src = (("hlstm_mma_kernel", "hlstm_mma.cu") if mode == "hlstm" else
+                                   ("recur_mma_kernel", "recur_mma.cu") if info.get("recur_register_resident")
                                    else ("recur_kernel", "recur.cu"))
         traffic = measured_traffic(kernel_name, args.workload, kernel_src)
         line = {

@@ -52,3 +52,39 @@ def test_hlstm_rejects_what_it_cannot_serve():
     with pytest.raises(pkg.LstmError) as e:
         pkg.HLSTM(weights, layers=1, in_dim=8, hidden=16, gate_hidden=16, dtype="fp32", max_T=2, max_B=1)
     assert e.value.code == pkg.LSTM_ERR_UNSUPPORTED
+
+
+def test_hlstm_withheld_words_end_in_a_timeout_status(oracle):
+    """Both exchanges of the H-LSTM step (hidden-layer values, h) are bounded waits: a CTA that withholds
+    its words makes the call end with LSTM_ERR_TIMEOUT, and the handle works again afterwards."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = wl.Workload("hlstm_timeout", 1, False, 24, 200, 6, 2, "bf16", 0.2, seed=77)
+    weights, x = wl.make_hlstm(w, 160)
+    ref = oracle.forward_hlstm(weights, x, layers=1, bidir=False, hidden=200, gate_hidden=160)
+    m = pkg.HLSTM(weights, layers=1, in_dim=24, hidden=200, gate_hidden=160, dtype="bf16", max_T=w.T, max_B=w.B)
+    xd = torch.from_numpy(x).cuda()
+    m.selftest_timeout(3, 2_000_000)
+    m.forward(xd)
+    assert m.status() == pkg.LSTM_ERR_TIMEOUT
+    m.selftest_timeout(-1)
+    y, hT, cT = m.forward(xd)
+    m.check()
+    assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", "after the timeout")
+    m.close()
+
+
+def test_hlstm_chunked_calls_carry_state(oracle):
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = wl.Workload("hlstm_chunks", 2, False, 30, 96, 10, 2, "bf16", 0.2, seed=78)
+    weights, x = wl.make_hlstm(w, 80)
+    ref = oracle.forward_hlstm(weights, x, layers=2, bidir=False, hidden=96, gate_hidden=80)
+    m = pkg.HLSTM(weights, layers=2, in_dim=30, hidden=96, gate_hidden=80, dtype="bf16", max_T=8, max_B=2)
+    xd = torch.from_numpy(x).cuda()
+    y1, h, c = m.forward(xd[:4].contiguous())
+    y2, h, c = m.forward(xd[4:].contiguous(), h, c)
+    m.check()
+    got = (torch.cat([y1, y2]).cpu().numpy(), h.cpu().numpy(), c.cpu().numpy())
+    assert_close(got, ref, "bf16", "chunked")
+    m.close()
