@@ -147,6 +147,17 @@ LSTM_API int lstm_forward(lstm_handle *h, const float *x, int T, int B, const fl
 LSTM_API int lstm_forward_host(lstm_handle *h, const float *x, int T, int B, const float *h0, const float *c0,
                       float *y, float *hT, float *cT, void *cuda_stream);
 
+/*
+ * The input projection of the first layer on its own (the x_t half of W [x_t, h_{t-1}] + b for all
+ * timesteps at once; the dense-versus-sparse matrix product the paper times in Section 3, Figures 1, 2):
+ *     g[t,b,d,q*Hg + j] = bias_q[j] + sum_k Wx_{d,q}[j,k] x[t,b,k]
+ * x [T,B,in_dim] and g [T,B,D,4*Hg] are DEVICE pointers (Hg = hidden, or gate_hidden for an H-LSTM handle
+ * where the rows are those of Ux and the bias is a); gate blocks i,f,g,o.  Runs the same staging and
+ * projection kernels as lstm_forward (tensor-core, CUDA-core or CSR according to the handle) plus a small
+ * re-layout kernel; enqueued on cuda_stream without synchronising.  0 <= T <= max_T, 0 <= B <= max_B.
+ */
+LSTM_API int lstm_input_projection(lstm_handle *h, const float *x, int T, int B, float *g, void *cuda_stream);
+
 /* Synchronises the stream last used with the handle and returns LSTM_OK or the recorded device
  * status (LSTM_ERR_TIMEOUT ...); the recorded status is cleared. */
 LSTM_API int lstm_status(lstm_handle *h);

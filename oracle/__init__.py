@@ -3,4 +3,4 @@
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this package; the
 CUDA library and its Python binding never do, and this package never imports them.
 """
-from .lstm_oracle import build, forward, forward_hlstm, threads, dense_to_csr  # noqa: F401
+from .lstm_oracle import build, forward, forward_hlstm, input_projection, threads, dense_to_csr  # noqa: F401

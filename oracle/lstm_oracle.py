@@ -110,6 +110,33 @@ def forward_hlstm(weights, x, h0=None, c0=None, *, layers: int, bidir: bool, hid
     return y, hT, cT
 
 
+def input_projection(weights, x, *, bidir: bool, hidden: int):
+    """The input half of the first layer's gate pre-activations for every position, written out as its
+    definition in float64 (Section 4: the x_t part of W [x_t, h_{t-1}] + b):
+    g[t,b,d,q*H+j] = b_q[j] + sum_k (Wx (x) Msk)[q*H+j,k] x[t,b,k].  ``weights``: the first layer's dict
+    per direction (``wx``, optional ``b``, ``mask_x``, or ``wx_csr``).  Returns [T,B,D,4H] float64."""
+    x = np.asarray(x, dtype=np.float64)
+    T, B, in_dim = x.shape
+    D, H = (2 if bidir else 1), int(hidden)
+    g = np.zeros((T, B, D, 4 * H), dtype=np.float64)
+    for d in range(D):
+        w = weights[d]
+        if w.get("wx_csr") is not None:
+            rp, col, val = w["wx_csr"]
+            wx = np.zeros((4 * H, in_dim), dtype=np.float64)
+            for r in range(4 * H):
+                wx[r, np.asarray(col[rp[r]:rp[r + 1]])] = np.asarray(val[rp[r]:rp[r + 1]], dtype=np.float64)
+        else:
+            wx = np.asarray(w["wx"], dtype=np.float64)
+            if w.get("mask_x") is not None:
+                wx = wx * (np.asarray(w["mask_x"]) != 0)
+        if wx.shape != (4 * H, in_dim):
+            raise ValueError(f"bad wx shape {wx.shape}")
+        bias = np.asarray(w["b"], dtype=np.float64) if w.get("b") is not None else np.zeros(4 * H)
+        g[:, :, d, :] = x @ wx.T + bias
+    return g
+
+
 def threads() -> int:
     """Number of OpenMP threads the oracle will use."""
     return int(_load().lstm_oracle_threads())

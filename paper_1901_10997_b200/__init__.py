@@ -5,7 +5,7 @@ arguments.  There is no CPU fallback: if the shared library is missing or no CUD
 the calls raise.
 """
 from .binding import (LSTM, HLSTM, LstmError, hlstm_create, lib_path, load_library, lstm_create, lstm_destroy,  # noqa: F401
-                      lstm_forward, lstm_forward_host, lstm_forward_noalloc, lstm_info, lstm_last_error,
+                      lstm_forward, lstm_forward_host, lstm_input_projection, lstm_forward_noalloc, lstm_info, lstm_last_error,
                       lstm_profile_enable, lstm_profile_read, lstm_selftest_timeout, lstm_status,
                       LSTM_F32, LSTM_BF16W_F32S, LSTM_DENSE, LSTM_CSR, LSTM_OK, LSTM_ERR_INVALID,
                       LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT,

@@ -56,6 +56,8 @@ def load_library():
         lib.hlstm_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, vp, ci, ci, vp]
         lib.lstm_forward.restype = ci
         lib.lstm_forward.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, vp, vp]
+        lib.lstm_input_projection.restype = ci
+        lib.lstm_input_projection.argtypes = [vp, vp, ci, ci, vp, vp]
         lib.lstm_forward_host.restype = ci
         lib.lstm_forward_host.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, vp, vp]
         lib.lstm_status.restype = ci
@@ -103,6 +105,10 @@ def hlstm_create(layers, in_dim, hidden, gate_hidden, bidir, dtype, weights_ptr,
 def lstm_forward(handle, x, T, B, h0, c0, y, hT, cT, stream=0):
     return load_library().lstm_forward(handle, x or None, T, B, h0 or None, c0 or None, y or None,
                                        hT or None, cT or None, stream or None)
+
+
+def lstm_input_projection(handle, x, T, B, g, stream=0):
+    return load_library().lstm_input_projection(handle, x or None, T, B, g or None, stream or None)
 
 
 def lstm_forward_host(handle, x, T, B, h0, c0, y, hT, cT, stream=0):
@@ -250,6 +256,17 @@ class LSTM:
                                  y.data_ptr(), hT.data_ptr() if hT is not None else 0,
                                  cT.data_ptr() if cT is not None else 0, st))
         return y, hT, cT
+
+    def input_projection(self, x, *, out=None, stream=None):
+        """First layer's input projection alone: x CUDA float32 [T,B,in_dim] -> [T,B,D,4*Hg] (gate blocks i,f,g,o)."""
+        import torch
+        T, B, _ = x.shape
+        hg = getattr(self, "gate_hidden", None) or self.hidden
+        if out is None:
+            out = torch.empty((T, B, self.dirs, 4 * hg), dtype=torch.float32, device=x.device)
+        st = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._check(lstm_input_projection(self._handle, x.data_ptr(), T, B, out.data_ptr(), st))
+        return out
 
     def forward_host(self, x, h0=None, c0=None, *, y=None, hT=None, cT=None, stream=0):
         """Host-buffer call: numpy arrays or CPU (ideally pinned) torch tensors in and out."""

@@ -760,6 +760,54 @@ static int record(lstm_handle *h, int kind, cudaStream_t st)
     return cudaEventRecord(h->ev[h->ev_used++], st) != cudaSuccess;
 }
 
+// Input staging (layer 0, tensor-core path) and projection of layer l for M rows into h->G; *nsplit receives
+// the number of split-K planes written.  x: the call's input (layer 0 only), Xf: fp32 activations of the layer.
+static int run_projection(lstm_handle *h, int l, const float *x, const float *Xf, int M, int N, int *nsplit_out, cudaStream_t st)
+{
+    Layer &ly = h->layers[l];
+    const bool bf16 = h->dtype == LSTM_BF16W_F32S;
+    const bool csr = h->exec_mode == LSTM_CSR;
+    cudaError_t e = cudaSuccess;
+    int nsplit = 1;
+    // ---- input staging + projection
+    if (csr) {
+        if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        e = launch_proj_csr(Xf, ly.wx_rowptr, ly.wx_ent, ly.bias, h->G, M, N, ly.in_l, !bf16, st);
+        ++h->last_launches;
+        if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+    } else if (h->use_tc) {
+        __nv_bfloat16 *xb = l == 0 ? h->xb0 : h->xbn[(l - 1) & 1];
+        if (l == 0) {
+            if (record(h, LSTM_K_STAGE, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_stage_bf16(x, xb, (long long)h->max_T * h->max_B * h->ld0, M, h->in_dim, h->ld0, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "staging launch failed: %s", cudaGetErrorString(e));
+        }
+        if (ly.plan_M != M) {
+            char msg[256];
+            const long long plane = (long long)h->max_T * h->max_B * ly.ldk;
+            if (proj_tc_plan(&ly.plan, (const __nv_bfloat16 *)ly.wx, xb, xb + plane, M, N, ly.in_l, ly.ldk, h->sm_count, msg, sizeof msg))
+                return fail(h, LSTM_ERR_CUDA, "tensor-core projection plan failed: %s", msg);
+            ly.plan_M = M;
+        }
+        nsplit = ly.plan.nsplit;
+        if ((size_t)nsplit * M * N > h->G_cap) return fail(h, LSTM_ERR_CUDA, "internal: projection workspace too small");
+        if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        e = launch_proj_tc(ly.plan, ly.bias, h->G, h->status_dev, st);
+        ++h->last_launches;
+        if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+    } else {
+        if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        e = launch_proj_simt(Xf, ly.wx, bf16, ly.ldk, ly.bias, h->G, M, N, ly.in_l, st);
+        ++h->last_launches;
+        if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+    }
+    if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "projection launch failed (layer %d): %s", l, cudaGetErrorString(e));
+    *nsplit_out = nsplit;
+    return LSTM_OK;
+}
+
 int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, const float *c0,
                  float *y, float *hT, float *cT, void *cuda_stream)
 {
@@ -805,40 +853,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         const int N = D * 4 * (h->Hh ? h->Hh : H);      // H-LSTM: the projection feeds the hidden layers
         int nsplit = 1;
         // ---- input staging + projection
-        if (csr) {
-            if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-            e = launch_proj_csr(Xf, ly.wx_rowptr, ly.wx_ent, ly.bias, h->G, M, N, ly.in_l, !bf16, st);
-            ++h->last_launches;
-            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-        } else if (h->use_tc) {
-            __nv_bfloat16 *xb = l == 0 ? h->xb0 : h->xbn[(l - 1) & 1];
-            if (l == 0) {
-                if (record(h, LSTM_K_STAGE, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-                e = launch_stage_bf16(x, xb, (long long)h->max_T * h->max_B * h->ld0, M, h->in_dim, h->ld0, st);
-                ++h->last_launches;
-                if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-                if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "staging launch failed: %s", cudaGetErrorString(e));
-            }
-            if (ly.plan_M != M) {
-                char msg[256];
-                const long long plane = (long long)h->max_T * h->max_B * ly.ldk;
-                if (proj_tc_plan(&ly.plan, (const __nv_bfloat16 *)ly.wx, xb, xb + plane, M, N, ly.in_l, ly.ldk, h->sm_count, msg, sizeof msg))
-                    return fail(h, LSTM_ERR_CUDA, "tensor-core projection plan failed: %s", msg);
-                ly.plan_M = M;
-            }
-            nsplit = ly.plan.nsplit;
-            if ((size_t)nsplit * M * N > h->G_cap) return fail(h, LSTM_ERR_CUDA, "internal: projection workspace too small");
-            if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-            e = launch_proj_tc(ly.plan, ly.bias, h->G, h->status_dev, st);
-            ++h->last_launches;
-            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-        } else {
-            if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-            e = launch_proj_simt(Xf, ly.wx, bf16, ly.ldk, ly.bias, h->G, M, N, ly.in_l, st);
-            ++h->last_launches;
-            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-        }
-        if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "projection launch failed (layer %d): %s", l, cudaGetErrorString(e));
+        { const int prc = run_projection(h, l, l == 0 ? x : nullptr, Xf, M, N, &nsplit, st); if (prc != LSTM_OK) return prc; }
 
         // ---- recurrence
         if (h->Hh) {
@@ -925,6 +940,27 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
         if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
     }
+    return LSTM_OK;
+}
+
+int lstm_input_projection(lstm_handle *h, const float *x, int T, int B, float *g, void *cuda_stream)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    if (T < 0 || B < 0 || T > h->max_T || B > h->max_B)
+        return fail(h, LSTM_ERR_INVALID, "T=%d B=%d outside [0,%d] x [0,%d]", T, B, h->max_T, h->max_B);
+    if (T == 0 || B == 0) return LSTM_OK;
+    if (!x || !g) return fail(h, LSTM_ERR_INVALID, "x and g must not be NULL");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    h->last_stream = st;
+    h->ev_used = 0;
+    h->last_launches = 0;
+    const int M = T * B, Hg = h->Hh ? h->Hh : h->H, N = h->D * 4 * Hg;
+    int nsplit = 1;
+    const int rc = run_projection(h, 0, x, x, M, N, &nsplit, st);
+    if (rc != LSTM_OK) return rc;
+    cudaError_t e = launch_proj_export(h->G, nsplit, (long long)M * N, g, M, h->D, Hg, st);
+    ++h->last_launches;
+    if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "export launch failed: %s", cudaGetErrorString(e));
     return LSTM_OK;
 }
 

@@ -139,6 +139,11 @@ struct CsrEntry { float val; int col; };
 cudaError_t launch_proj_csr(const float *X, const int *rowptr, const CsrEntry *ent,
                             const float *bias, float *G, int M, int N, int K, bool f64_acc, cudaStream_t st);
 
+// out[m][d][q][j] = sum over split planes of G[split][m][d][j][q]: the projection in the public layout
+// (gate blocks i,f,g,o of Hg rows per direction) from the internal unit-major one
+cudaError_t launch_proj_export(const float *G, int nsplit, long long split_stride, float *out, long long M, int D, int Hg,
+                               cudaStream_t st);
+
 // Tensor-core projection (tcgen05 + TMEM + TMA).  A = packed weights [N][ldk] bf16 (K-major),
 // activations [M][ldk] as two bf16 planes (hi, lo); writes G[split][M][N] fp32 (+bias on split 0).
 struct ProjTcPlan {

@@ -126,7 +126,34 @@ __global__ void __launch_bounds__(256) proj_csr_kernel(const float *__restrict__
     }
 }
 
+__global__ void proj_export_kernel(const float *__restrict__ G, int nsplit, long long split_stride,
+                                   float *__restrict__ out, long long M, int D, int Hg)
+{
+    const long long total = M * D * 4 * Hg;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        // i enumerates the public layout [m][d][q][j]
+        const int j = (int)(i % Hg);
+        const int q = (int)((i / Hg) % 4);
+        const long long md = i / (4 * Hg);
+        const long long src = (md * Hg + j) * 4 + q;
+        float v = 0.0f;
+        for (int sp = 0; sp < nsplit; ++sp) v += G[sp * split_stride + src];
+        out[i] = v;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_proj_export(const float *G, int nsplit, long long split_stride, float *out, long long M, int D, int Hg,
+                               cudaStream_t st)
+{
+    const long long total = M * D * 4 * Hg;
+    if (total == 0) return cudaSuccess;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 16) blocks = 148LL * 16;
+    proj_export_kernel<<<(int)blocks, 256, 0, st>>>(G, nsplit, split_stride, out, M, D, Hg);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_stage_bf16(const float *x, __nv_bfloat16 *xb, long long plane, long long M, int K, int ld,
                               cudaStream_t st)

@@ -227,3 +227,27 @@ def test_withheld_exchange_words_end_in_a_timeout_status_not_a_hang(oracle, dtyp
     m.check()
     assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, dtype, "after the timeout")
     m.close()
+
+
+# ---------------------------------------------------------------- the input projection on its own
+@pytest.mark.parametrize("case", [("bf16", "dense", 1.0), ("bf16", "dense", 0.1), ("bf16", "csr", 0.1), ("fp32", "dense", 1.0),
+                                  ("fp32", "csr", 0.3)], ids=lambda c: f"{c[0]}-{c[1]}-{c[2]}")
+@pytest.mark.parametrize("shape", [(1, 7, 9, 3, 2), (2, 200, 136, 5, 3), (1, 1500, 375, 16, 1), (2, 1312, 200, 40, 4)],
+                         ids=lambda s: f"D{s[0]}_in{s[1]}_H{s[2]}_T{s[3]}_B{s[4]}")
+def test_input_projection_alone(oracle, case, shape):
+    """Tensor-core, CUDA-core and CSR projections against the matrix product written out, ragged in every
+    dimension (rows, columns, K tail), with split-K (short sequences) and without."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    dtype, mode, density = case
+    D, in_dim, H, T, B = shape
+    w = wl.Workload("proj", 1, D == 2, in_dim, H, T, B, dtype, 0.2, density=density, seed=in_dim + H)
+    weights, x = wl.make(w)
+    ref = oracle.input_projection(weights, x, bidir=D == 2, hidden=H)
+    m = pkg.LSTM(weights, layers=1, in_dim=in_dim, hidden=H, bidir=D == 2, dtype=dtype, exec_mode=mode, max_T=T, max_B=B)
+    g = m.input_projection(torch.from_numpy(x).cuda())
+    m.check()
+    floored, scaled = wl.rel_err(g.cpu().numpy(), ref)
+    # one rounding of each activation term (bf16 hi + lo, about 2^-17) or fp32 storage of the result
+    assert scaled <= (1e-4 if dtype == "bf16" else 1e-6), (floored, scaled)
+    m.close()

@@ -410,3 +410,37 @@ def test_planted_mistakes_are_caught(oracle, tmp_path):
         assert src.count(old) >= 1, f"mutation target not found: {name}"
         worst = _run_pins_on(compile_variant(src.replace(old, new, 1), f"mut{n}"))
         assert worst > 1e-6, f"planted mistake not caught: {name}"
+
+
+# ---------------------------------------------------------------- the projection on its own
+def test_input_projection_definition_and_its_tie_to_the_cell(oracle):
+    """oracle.input_projection is the matrix product written out; it is pinned by explicit loops on a tiny
+    case and by the cell oracle: with Wh = 0 and zero initial state, one step gives
+    h = sigmoid(g_o) tanh(sigmoid(g_i) tanh(g_g)) from the projection values alone."""
+    rng = np.random.default_rng(77)
+    H, in_dim, T, B = 3, 4, 2, 2
+    ws = rand_weights(rng, 1, 2, in_dim, H, scale=0.8)
+    mask = (rng.random((4 * H, in_dim)) < 0.6).astype(np.uint8)
+    ws[1]["mask_x"] = mask
+    x = rng.standard_normal((T, B, in_dim))
+    g = oracle.input_projection(ws, x, bidir=True, hidden=H)
+    for d in range(2):
+        for t in range(T):
+            for b in range(B):
+                for r in range(4 * H):
+                    acc = float(ws[d]["b"][r])
+                    for k in range(in_dim):
+                        keep = 1.0 if (d == 0 or mask[r, k]) else 0.0
+                        acc += float(ws[d]["wx"][r, k]) * keep * x[t, b, k]
+                    assert g[t, b, d, r] == pytest.approx(acc, rel=1e-13, abs=1e-15)
+    # tie to the cell: first step of the forward direction, no recurrent weights
+    w0 = {**ws[0], "wh": np.zeros((4 * H, H), np.float32)}
+    y, _, _ = oracle.forward([w0], x[:1], layers=1, bidir=False, hidden=H)
+    for b in range(B):
+        for j in range(H):
+            gi, gg, go = g[0, b, 0, j], g[0, b, 0, 2 * H + j], g[0, b, 0, 3 * H + j]
+            assert y[0, b, j] == pytest.approx(sig(go) * math.tanh(sig(gi) * math.tanh(gg)), rel=1e-13)
+    # CSR description of the same matrix
+    csr = [{"wx_csr": oracle.dense_to_csr(ws[1]["wx"], mask), "b": ws[1]["b"]}]
+    g_csr = oracle.input_projection(csr, x, bidir=False, hidden=H)
+    assert np.array_equal(g_csr[:, :, 0], g[:, :, 1])
