@@ -13,6 +13,7 @@ data path, N sequences per step.
 Other modes:
     --impl reference     time the fp64 CPU oracle on the same workload (host cores only)
     --sweep              latency vs hidden size (H = 128..2048 step 8) with the LHP analysis
+    --matmul-sweep       dense (tensor-core) vs sparse (CSR) matrix product at batch 16, d = 128..2048
     --workload NAME      cfg1 | cfg2 | cfg2_b20 | cfg4_10 | cfg4_05 | cfg4_10_csr | cfg4_05_csr |
                          cfg5 | cfg5_b16 (default cfg2)
 """
@@ -444,6 +445,50 @@ def run_sweep(args):
     print(json.dumps({k: v for k, v in res.items() if k != "points"}))
 
 
+def run_matmul_sweep(args):
+    """The paper's Figures 1 and 2 on this GPU: one square matrix W [d x d] times a batch of 16 dense columns,
+    dense (tensor-core projection, bf16 weights) against sparse (CSR projection over the surviving weights)
+    at 90 % and 95 % sparsity, d = 128 .. 2048.  Timed with the library's per-kernel events (staging +
+    projection kernels), L2 flushed between calls."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    dev = torch.device("cuda", 0)
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    outdir = ROOT / "gpurun_out"
+    outdir.mkdir(exist_ok=True)
+    rows = []
+    for dsz in range(128, 2048 + 1, 64):
+        H = dsz // 4
+        row = {"d": dsz}
+        for label, density, mode in (("dense_tc", 1.0, "dense"), ("csr_10", 0.10, "csr"), ("csr_05", 0.05, "csr")):
+            w = wl.Workload(f"matmul_d{dsz}", 1, False, dsz, H, 16, 1, "bf16", 1.0 / np.sqrt(dsz), density=density,
+                            seed=wl.SEED_BASE + dsz)
+            weights, x = wl.make(w)
+            m = pkg.LSTM(weights, layers=1, in_dim=dsz, hidden=H, dtype="bf16", exec_mode=mode, max_T=16, max_B=1)
+            xd = torch.from_numpy(x).to(dev)
+            out = torch.empty((16, 1, 1, 4 * H), device=dev)
+            m.profile_enable(True)
+            ts = []
+            for i in range(args.steps + max(args.warmup, 3)):
+                flush_l2(flush_buf)
+                m.input_projection(xd, out=out)
+                _n, t = m.profile_read()
+                if i >= max(args.warmup, 3):
+                    ts.append((t[pkg.LSTM_K_STAGE] + t[pkg.LSTM_K_PROJ]) * 1e3)
+            m.check()
+            if args.sweep_parity:
+                import oracle
+                ref = oracle.input_projection(weights, x, bidir=False, hidden=H)
+                row[label + "_err"] = wl.rel_err(out.cpu().numpy().reshape(ref.shape), ref)[1]
+            m.close()
+            row[label + "_us"] = float(np.percentile(ts, 50))
+        rows.append(row)
+        print(json.dumps(row), file=sys.stderr, flush=True)
+    (outdir / "matmul_sweep.json").write_text(json.dumps({"batch": 16, "steps": args.steps, "points": rows}, indent=1))
+    wins = sum(1 for r in rows if r["csr_05_us"] < r["dense_tc_us"])
+    print(json.dumps({"points": len(rows), "sparse_95_faster_than_dense_at": wins}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -453,6 +498,7 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--matmul-sweep", action="store_true")
     ap.add_argument("--sweep-sizes", default="")
     ap.add_argument("--sweep-parity", action="store_true")
     args = ap.parse_args()
@@ -460,6 +506,8 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+    elif args.matmul_sweep:
+        run_matmul_sweep(args)
     else:
         run_gpu(args)
 

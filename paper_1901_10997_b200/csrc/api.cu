@@ -571,6 +571,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                             : h->use_mma ? recur_mma_prepare(h->mma_mt, h->mma_nkr, h->mma_nw, h->smem_optin - 64)
                                          : recur_dense_prepare(h->smem_optin - 64);
         if (e == cudaSuccess && h->use_tc) e = proj_tc_prepare();
+        if (e == cudaSuccess && csr) e = proj_csr_prepare(h->smem_optin - 64);
         if (e != cudaSuccess) rc = fail(h, LSTM_ERR_CUDA, "kernel set-up failed: %s", cudaGetErrorString(e));
     }
     if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)

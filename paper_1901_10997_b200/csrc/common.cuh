@@ -136,6 +136,7 @@ cudaError_t launch_proj_simt(const float *X, const void *W, bool bf16_weights, i
 
 // G[m][n] = sum_e val[e] * X[m][col[e]] + bias[n] over CSR row n (entries {val,col} pairs)
 struct CsrEntry { float val; int col; };
+cudaError_t proj_csr_prepare(int max_smem);   // raises the dynamic shared-memory limit once
 cudaError_t launch_proj_csr(const float *X, const int *rowptr, const CsrEntry *ent,
                             const float *bias, float *G, int M, int N, int K, bool f64_acc, cudaStream_t st);
 

@@ -83,6 +83,7 @@ __global__ void __launch_bounds__(256) proj_simt_kernel(const float *__restrict_
 // CSR projection: a CTA stages MT = 8 activation rows (transposed so that the 8 values of one column
 // are contiguous) and its warps walk CSR rows; lanes stride over a row's entries.
 constexpr int kCsrMT = 8;
+constexpr int kCsrUnroll = 8;
 template <typename AT>
 __global__ void __launch_bounds__(256) proj_csr_kernel(const float *__restrict__ X, const int *__restrict__ rowptr,
                                                        const CsrEntry *__restrict__ ent,
@@ -91,9 +92,14 @@ __global__ void __launch_bounds__(256) proj_csr_kernel(const float *__restrict__
 {
     extern __shared__ __align__(16) float xt[];          // [K][8]
     const int m0 = blockIdx.y * kCsrMT;
-    for (int i = threadIdx.x; i < K * kCsrMT; i += blockDim.x) {
-        const int mm = i / K, k = i - mm * K;             // coalesced over k
-        xt[k * kCsrMT + mm] = (m0 + mm < M) ? X[(size_t)(m0 + mm) * K + k] : 0.0f;
+    // a thread fetches one column of all eight rows at once (eight loads in flight, coalesced over the
+    // threads) and stores them as the 32 contiguous bytes the row walk reads back
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float v[kCsrMT];
+#pragma unroll
+        for (int mm = 0; mm < kCsrMT; ++mm) v[mm] = (m0 + mm < M) ? X[(size_t)(m0 + mm) * K + k] : 0.0f;
+        *reinterpret_cast<float4 *>(xt + (size_t)k * kCsrMT) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4 *>(xt + (size_t)k * kCsrMT + 4) = make_float4(v[4], v[5], v[6], v[7]);
     }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -103,15 +109,26 @@ __global__ void __launch_bounds__(256) proj_csr_kernel(const float *__restrict__
         AT acc[kCsrMT];
 #pragma unroll
         for (int i = 0; i < kCsrMT; ++i) acc[i] = (AT)0;
-        for (int e = rowptr[r] + lane; e < rowptr[r + 1]; e += 32) {
-            const CsrEntry en = ent[e];
-            const float4 a = *reinterpret_cast<const float4 *>(xt + (size_t)en.col * kCsrMT);
-            const float4 b = *reinterpret_cast<const float4 *>(xt + (size_t)en.col * kCsrMT + 4);
-            const AT v = (AT)en.val;
-            acc[0] = fma(v, (AT)a.x, acc[0]); acc[1] = fma(v, (AT)a.y, acc[1]);
-            acc[2] = fma(v, (AT)a.z, acc[2]); acc[3] = fma(v, (AT)a.w, acc[3]);
-            acc[4] = fma(v, (AT)b.x, acc[4]); acc[5] = fma(v, (AT)b.y, acc[5]);
-            acc[6] = fma(v, (AT)b.z, acc[6]); acc[7] = fma(v, (AT)b.w, acc[7]);
+        // entries of a row are fetched eight lane-strides at a time, so that one trip to memory covers a
+        // row of up to 256 survivors instead of one trip per 32
+        const int e_end = rowptr[r + 1];
+        for (int e0 = rowptr[r] + lane; e0 < e_end; e0 += 32 * kCsrUnroll) {
+            CsrEntry en[kCsrUnroll];
+#pragma unroll
+            for (int u = 0; u < kCsrUnroll; ++u) {
+                const int e = e0 + 32 * u;
+                en[u] = e < e_end ? ent[e] : CsrEntry{0.0f, 0};
+            }
+#pragma unroll
+            for (int u = 0; u < kCsrUnroll; ++u) {
+                const float4 a = *reinterpret_cast<const float4 *>(xt + (size_t)en[u].col * kCsrMT);
+                const float4 b = *reinterpret_cast<const float4 *>(xt + (size_t)en[u].col * kCsrMT + 4);
+                const AT v = (AT)en[u].val;
+                acc[0] = fma(v, (AT)a.x, acc[0]); acc[1] = fma(v, (AT)a.y, acc[1]);
+                acc[2] = fma(v, (AT)a.z, acc[2]); acc[3] = fma(v, (AT)a.w, acc[3]);
+                acc[4] = fma(v, (AT)b.x, acc[4]); acc[5] = fma(v, (AT)b.y, acc[5]);
+                acc[6] = fma(v, (AT)b.z, acc[6]); acc[7] = fma(v, (AT)b.w, acc[7]);
+            }
         }
 #pragma unroll
         for (int i = 0; i < kCsrMT; ++i)
@@ -179,18 +196,20 @@ cudaError_t launch_proj_simt(const float *X, const void *W, bool bf16, int ldw, 
     return cudaGetLastError();
 }
 
+cudaError_t proj_csr_prepare(int max_smem)
+{
+    cudaError_t e = cudaFuncSetAttribute(proj_csr_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(proj_csr_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+}
+
 cudaError_t launch_proj_csr(const float *X, const int *rowptr, const CsrEntry *ent, const float *bias,
                             float *G, int M, int N, int K, bool f64_acc, cudaStream_t st)
 {
     if (M == 0 || N == 0) return cudaSuccess;
     const size_t smem = (size_t)K * kCsrMT * sizeof(float);
-    if (smem > 48 * 1024) {
-        cudaError_t e = f64_acc ? cudaFuncSetAttribute(proj_csr_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                                : cudaFuncSetAttribute(proj_csr_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
     const int mtiles = (M + kCsrMT - 1) / kCsrMT;
-    int ctas_x = max(1, (148 * 2) / mtiles);
+    int ctas_x = max(1, (148 * 4) / mtiles);      // about four CTAs per SM: a warp walks few rows, one trip to memory each
     int rows_per_cta = max(8, (N + ctas_x - 1) / ctas_x);
     ctas_x = (N + rows_per_cta - 1) / rows_per_cta;
     dim3 grid(ctas_x, mtiles);
