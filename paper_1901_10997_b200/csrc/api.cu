@@ -643,7 +643,7 @@ int hlstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int gate
     h->smem_optin = (int)prop.sharedMemPerBlockOptin;
     h->last_stream = st;
     h->Hp8 = round_up(H, 8); h->Hs = round_up(H, 256);
-    h->ncta_dir = std::max(1, std::min(h->sm_count / D, std::min(H, Hh)));
+    h->ncta_dir = std::max(1, std::min(h->sm_count / D, std::max(H, Hh)));   // a CTA may own no unit of the narrower side
     h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
     h->threads = 512;
     h->use_tc = true;

@@ -88,3 +88,21 @@ def test_hlstm_chunked_calls_carry_state(oracle):
     got = (torch.cat([y1, y2]).cpu().numpy(), h.cpu().numpy(), c.cpu().numpy())
     assert_close(got, ref, "bf16", "chunked")
     m.close()
+
+
+def _fuzz_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    return [dict(L=int(rng.integers(1, 3)), bidir=bool(rng.integers(0, 2)), in_dim=int(rng.integers(1, 150)),
+                 H=int(rng.choice([rng.integers(1, 50), rng.integers(50, 600)])),
+                 Hh=int(rng.choice([rng.integers(1, 50), rng.integers(50, 600)])),
+                 T=int(rng.integers(1, 8)), B=int(rng.integers(1, 5)), seed=500 + i) for i in range(n)]
+
+
+@pytest.mark.parametrize("c", _fuzz_cases(16, 77), ids=lambda c: "L{L}D{d}_in{in_dim}_H{H}_Hh{Hh}_T{T}_B{B}".format(d=1 + c["bidir"], **c))
+def test_hlstm_random_shapes(oracle, c):
+    scale = min(0.3, 2.0 / np.sqrt(max(c["H"], c["Hh"]) + c["in_dim"]))
+    w = wl.Workload("hfuzz", c["L"], c["bidir"], c["in_dim"], c["H"], c["T"], c["B"], "bf16", scale, seed=c["seed"])
+    weights, x = wl.make_hlstm(w, c["Hh"])
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward_hlstm(weights, x, h0, c0, layers=c["L"], bidir=c["bidir"], hidden=c["H"], gate_hidden=c["Hh"])
+    assert_close(run(w, c["Hh"], weights, x, h0, c0), ref, "bf16", "hlstm fuzz")

@@ -251,3 +251,30 @@ def test_input_projection_alone(oracle, case, shape):
     # one rounding of each activation term (bf16 hi + lo, about 2^-17) or fp32 storage of the result
     assert scaled <= (1e-4 if dtype == "bf16" else 1e-6), (floored, scaled)
     m.close()
+
+
+# ---------------------------------------------------------------- seeded random shapes
+def _fuzz_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        H = int(rng.choice([rng.integers(1, 40), rng.integers(40, 300), rng.integers(300, 900)]))
+        cases.append(dict(L=int(rng.integers(1, 3)), bidir=bool(rng.integers(0, 2)), in_dim=int(rng.integers(1, 200)), H=H,
+                          T=int(rng.integers(1, 10)), B=int(rng.integers(1, 10)), dtype=str(rng.choice(["bf16", "bf16", "fp32"])),
+                          mode=str(rng.choice(["dense", "dense", "csr"])), states=bool(rng.integers(0, 2)),
+                          density=float(rng.choice([1.0, 0.3])), seed=1000 + i))
+    return cases
+
+
+@pytest.mark.parametrize("c", _fuzz_cases(36, 2024), ids=lambda c: "L{L}D{d}_in{in_dim}_H{H}_T{T}_B{B}_{dtype}_{mode}".format(d=1 + c["bidir"], **c))
+def test_random_shapes(oracle, c):
+    """Shapes nobody picked by hand: every kernel variant (register-resident, shared-memory, CSR; staged and
+    polled exchange; tensor-core, CUDA-core and CSR projections) against the oracle."""
+    scale = min(0.3, 2.0 / np.sqrt(c["H"] + c["in_dim"]))
+    w = wl.Workload("fuzz", c["L"], c["bidir"], c["in_dim"], c["H"], c["T"], c["B"], c["dtype"], scale,
+                    density=c["density"], seed=c["seed"])
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w) if c["states"] else (None, None)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got = run_gpu(w, weights, x, h0, c0, exec_mode=c["mode"])
+    assert_close(got, ref, w.dtype, "fuzz")
