@@ -30,6 +30,8 @@ struct Layer {
     int *wh_ptr[2] = {nullptr, nullptr};   // CSR recurrence: padded entry offsets [4H+1]
     void *wh_ent[2] = {nullptr, nullptr};
     uint4 *wfrag[2] = {nullptr, nullptr};  // register-resident kernel: operand-A fragments
+    __nv_bfloat16 *wtc = nullptr;          // batched tensor-core kernel: [D * ncta * RA][ld64] rows 4*unit+gate per CTA
+    alignas(64) unsigned char tmap_wtc[128];
     uint4 *frag2[2] = {nullptr, nullptr};  // H-LSTM: fragments of the gate output matrices W
     float *bias_out = nullptr;             // H-LSTM: [D][H][4] bias of the gate pre-activations
     int csr_max_slice_entries = 0;     // largest per-CTA slice (entries, padded)
@@ -49,6 +51,11 @@ struct lstm_handle {
     // in shared memory, warps per CTA
     bool use_mma = false;
     int mma_mt = 0, mma_nkr = 0, mma_nks = 0, mma_nw = 0;
+    // batched tensor-core recurrence (more than four batch rows): weight-tile rows, K blocks, planes, stamps
+    bool use_tcb = false;
+    int tcb_RA = 0, tcb_nkb = 0, tcb_ld = 0, tcb_ldh = 0, tcb_mapN = 0;
+    __nv_bfloat16 *hplanes = nullptr; unsigned *tcb_flags = nullptr;
+    alignas(64) unsigned char tmap_planes[128];
     // H-LSTM cell: width of the hidden layer inside each gate (0: plain LSTM), pass-2 column tiles per warp
     int Hh = 0, hl_nkw2 = 0;
     unsigned long long *rxch = nullptr; size_t rxch_words = 0;
@@ -333,10 +340,10 @@ void free_all(lstm_handle *h)
     for (auto &ly : h->layers) {
         cudaFree(ly.wx); cudaFree(ly.bias); cudaFree(ly.wx_rowptr); cudaFree(ly.wx_ent);
         for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); cudaFree(ly.frag2[d]); }
-        cudaFree(ly.bias_out);
+        cudaFree(ly.bias_out); cudaFree(ly.wtc);
     }
     cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
-    cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->rxch); cudaFree(h->status_dev);
+    cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->rxch); cudaFree(h->hplanes); cudaFree(h->tcb_flags); cudaFree(h->status_dev);
     cudaFree(h->hx); cudaFree(h->hy); cudaFree(h->hh0); cudaFree(h->hc0); cudaFree(h->hhT); cudaFree(h->hcT);
     for (auto e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
@@ -399,6 +406,16 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
     plan_mma(h);
+    {   // batched tensor-core recurrence: available beside the register-resident kernel when the slice fits
+        const char *env = getenv("LSTM_B200_RECUR");
+        const int RA = round_up(4 * h->upc, 8), nkb = (H + 63) / 64;
+        if (h->use_mma && max_B > 4 && RA <= 128 && !(env && strcmp(env, "mma") == 0)) {
+            const int B = std::min(max_B, 32), N = round_up(2 * B, 16);
+            if (recur_tc_smem_bytes(RA, nkb, N, std::min(8, nkb), h->upc, B) <= (size_t)h->smem_optin - 256) {
+                h->use_tcb = true; h->tcb_RA = RA; h->tcb_nkb = nkb; h->tcb_ld = nkb * 64; h->tcb_ldh = round_up(H, 8);
+            }
+        }
+    }
     h->layers.resize(layers);
     if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
     h->spin_limit_default = h->spin_limit;
@@ -416,6 +433,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
         std::vector<float> bias_p((size_t)N, 0.0f);
         std::vector<uint16_t> wx16; std::vector<float> wx32;
         std::vector<int> px_rowptr; std::vector<CsrEntry> px_ent;
+        std::vector<uint16_t> tcb_rows;
         if (!csr) { if (bf16) wx16.assign((size_t)N * ly.ldk, 0); else wx32.assign((size_t)N * ly.ldk, 0.0f); }
         else px_rowptr.assign(N + 1, 0);
 
@@ -473,6 +491,20 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                     }
                     rc = upload(h, (uint32_t **)&ly.wfrag[d], f.data(), f.size() * 4, st, "recurrent weight fragments");
                     if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                    if (rc == LSTM_OK && h->use_tcb) {
+                        // the same slices as plain K-major rows for the tensor-core kernel's TMA tiles
+                        const size_t rows_dir = (size_t)h->ncta_dir * h->tcb_RA;
+                        if (d == 0) tcb_rows.assign((size_t)D * rows_dir * h->tcb_ld, 0);
+                        for (int c = 0; c < h->ncta_dir; ++c) {
+                            int u0, nu; unit_range_host(H, h->ncta_dir, c, u0, nu);
+                            for (int u = 0; u < nu; ++u)
+                                for (int q = 0; q < 4; ++q) {
+                                    const float *srow = m.data() + (size_t)(q * H + u0 + u) * H;
+                                    uint16_t *drow = tcb_rows.data() + ((size_t)d * rows_dir + (size_t)c * h->tcb_RA + 4 * u + q) * h->tcb_ld;
+                                    for (int k = 0; k < H; ++k) drow[k] = f32_to_bf16_rne(srow[k]);
+                                }
+                        }
+                    }
                 } else if (bf16) {
                     std::vector<uint16_t> p(n, 0);
                     for (int j = 0; j < H; ++j)
@@ -536,6 +568,11 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
         }
         if (rc) break;
         rc = upload(h, &ly.bias, bias_p.data(), bias_p.size() * 4, st, "bias");
+        if (rc == LSTM_OK && h->use_tcb && !tcb_rows.empty()) {
+            rc = upload(h, (uint16_t **)&ly.wtc, tcb_rows.data(), tcb_rows.size() * 2, st, "recurrent weight tiles");
+            if (rc == LSTM_OK && !recur_tc_encode_weights(ly.tmap_wtc, ly.wtc, (long long)D * h->ncta_dir * h->tcb_RA, h->tcb_ld, h->tcb_RA))
+                rc = fail(h, LSTM_ERR_CUDA, "tensor map of the recurrent weight tiles could not be encoded");
+        }
         if (rc == LSTM_OK && !csr)
             rc = bf16 ? upload(h, (uint16_t **)&ly.wx, wx16.data(), wx16.size() * 2, st, "input weights")
                       : upload(h, (float **)&ly.wx, wx32.data(), wx32.size() * 4, st, "input weights");
@@ -565,6 +602,10 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
         for (int i = 0; i < 2 && rc == LSTM_OK; ++i) rc = dev_alloc(h, &h->ybuf[i], Mmax * D * H * 4, false, st, "layer activations");
     h->xch_words = (size_t)D * 2 * max_B * H;
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->xch, h->xch_words * 8, true, st, "exchange buffer");
+    if (rc == LSTM_OK && h->use_tcb) {
+        rc = dev_alloc(h, &h->hplanes, (size_t)D * 2 * 64 * h->tcb_ldh * 2, true, st, "h planes");
+        if (rc == LSTM_OK) rc = dev_alloc(h, &h->tcb_flags, (size_t)D * h->ncta_dir * sizeof(unsigned), true, st, "stamps");
+    }
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
     if (rc == LSTM_OK) {
         cudaError_t e = csr ? recur_csr_prepare(h->smem_optin - 64)
@@ -572,6 +613,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                                          : recur_dense_prepare(h->smem_optin - 64);
         if (e == cudaSuccess && h->use_tc) e = proj_tc_prepare();
         if (e == cudaSuccess && csr) e = proj_csr_prepare(h->smem_optin - 64);
+        if (e == cudaSuccess && h->use_tcb) e = recur_tc_prepare(h->smem_optin - 256);
         if (e != cudaSuccess) rc = fail(h, LSTM_ERR_CUDA, "kernel set-up failed: %s", cudaGetErrorString(e));
     }
     if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)
@@ -845,6 +887,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
     if ((unsigned long long)h->stamp_next + (unsigned long long)L * T + 2ull >= 0xffffffffull) {
         if (cudaMemsetAsync(h->xch, 0, h->xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->rxch && cudaMemsetAsync(h->rxch, 0, h->rxch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
+        if (h->tcb_flags && cudaMemsetAsync(h->tcb_flags, 0, (size_t)D * h->ncta_dir * sizeof(unsigned), st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         h->stamp_next = 0;
     }
 
@@ -882,6 +925,41 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             const size_t smem = hlstm_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->hl_nkw2, h->upc, B);
             if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
             e = launch_hlstm_mma(m, h->mma_mt, h->mma_nkr, h->mma_nw, smem, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
+            continue;
+        }
+        if (h->use_tcb && B > 4 && B <= 32) {
+            RecurTcArgs m;
+            memset(&m, 0, sizeof m);
+            m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
+            m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16); m.stages = std::min(8, h->tcb_nkb);
+            m.tmem_cols = m.N <= 32 ? 32 : 64;
+            m.ldh = h->tcb_ldh;
+            m.stamp_base = h->stamp_next;
+            h->stamp_next += (unsigned)T + 1u;
+            m.spin_limit = h->spin_limit;
+            m.withhold_cta = h->withhold_cta;
+            m.G = h->G;
+            m.g_split_stride = (long long)M * N;
+            const size_t so = (size_t)l * D * B * H;
+            m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
+            m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
+            m.y = l == L - 1 ? y : h->ybuf[l & 1];
+            m.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
+            m.xb_ld = h->ldn;
+            m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
+            m.hbuf = h->hplanes; m.flags = h->tcb_flags;
+            m.status = h->status_dev;
+            if (h->tcb_mapN != m.N) {
+                if (!recur_tc_encode_planes(h->tmap_planes, h->hplanes, D, H, h->tcb_ldh, m.N))
+                    return fail(h, LSTM_ERR_CUDA, "tensor map of the h planes could not be encoded");
+                h->tcb_mapN = m.N;
+            }
+            const size_t smem = recur_tc_smem_bytes(m.RA, m.nkb, m.N, m.stages, h->upc, B);
+            if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_recur_tc(ly.tmap_wtc, h->tmap_planes, m, smem, st);
             ++h->last_launches;
             if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
             if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));

@@ -89,6 +89,42 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------------
+// Batched recurrent kernel on tcgen05 (bf16 weights, dense, more than four batch rows).  The CTA's slice of
+// Wh sits in shared memory as K-major 128-byte-swizzled tiles of RA rows (4 * units per CTA rounded up to 8)
+// per 64 columns; h travels through global memory as bf16 planes [D][2 parities][64 rows][ldh] (row 2b = hi,
+// 2b+1 = lo part of batch row b) and one stamp per producer CTA.
+// ---------------------------------------------------------------------------------------------------
+struct RecurTcArgs {
+    int H, B, T, D;
+    int ncta_dir;
+    int nsplit;
+    int RA, nkb;                // rows of a weight tile; 64-column K blocks
+    int N;                      // MMA N: 2 * B rounded up to 16
+    int stages;                 // depth of the operand ring
+    int tmem_cols;              // power of two >= max(32, N)
+    int ldh;                    // row stride of the planes (elements, multiple of 8)
+    unsigned stamp_base;
+    long long spin_limit;
+    int withhold_cta;
+    const float *G;
+    long long g_split_stride;
+    const float *h0, *c0;
+    float *hT, *cT;
+    float *y;
+    __nv_bfloat16 *xb_next;
+    long long xb_plane;
+    int xb_ld;
+    __nv_bfloat16 *hbuf;
+    unsigned *flags;            // [D][ncta_dir]
+    int *status;
+};
+size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int upc, int B);
+bool recur_tc_encode_weights(void *map128, const void *w, long long rows, int ld, int RA);
+bool recur_tc_encode_planes(void *map128, const void *hbuf, int D, int H, int ldh, int N);
+cudaError_t recur_tc_prepare(int max_smem);
+cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurTcArgs &a, size_t smem, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------
 // H-LSTM recurrent kernel (one ReLU hidden layer of width Hh inside each gate; bf16 weights, dense).
 // Pass 1 works on the four Uh_q [Hh x H] (hidden units split over the CTAs, fragments in registers and,
 // beyond nkr tiles per warp, in shared memory), pass 2 on the four W_q [H x Hh] (cell units split over the

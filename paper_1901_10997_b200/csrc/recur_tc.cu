@@ -1,0 +1,405 @@
+// Batched recurrent kernel for bf16 weights on the 5th-generation tensor cores: the serial half of the LSTM
+// forward pass (paper, Section 4, cell equations with zero hidden layers per gate)
+//     z = G[t] + Wh h_{t-1};  i,f,o = sigmoid(z_i,z_f,z_o), g = tanh(z_g);  c_t = f c_{t-1} + i g;
+//     h_t = o tanh(c_t)
+// for batches of more than four sequences, where the per-step product Wh_slice [4u x H] . h_{t-1} [H x B]
+// is a real (if skinny) matrix product and one tcgen05.mma chain per step replaces the ceil(B/4) passes of
+// the register-resident kernel.
+//
+// One cooperative launch runs all T steps of one layer (both directions on disjoint CTA groups).  A CTA
+// owns a contiguous range of hidden units; its slice of Wh (rows 4*unit + gate) is loaded ONCE by TMA into
+// shared memory as 128-byte-swizzled K-major tiles (one per 64 columns) and stays there.  h travels
+// between CTAs through global memory as the tensor cores want it: two bf16 planes per batch row (row 2b =
+// hi, row 2b+1 = lo, so products keep about 16 mantissa bits), K-major.  Per step:
+//   warp 0   polls one stamp per producer CTA (acquire loads, bounded), then streams the [2B x H] operand
+//            into a ring of shared-memory stages with TMA (64 columns per stage, zero fill at the tail);
+//   warp 1   issues M = 128, N = 2B (rounded up to 16), K = 16 tcgen05.mma instructions into one TMEM
+//            accumulator; the weight tile has only 4*units (<= 128) real rows: the rows beyond read whatever
+//            follows in shared memory and produce accumulator rows nobody reads;
+//   warps 2-5 read the accumulator rows of the CTA's units back (tcgen05.ld), add hi and lo columns, and
+//            finish the (unit, batch row) pairs: projection term, gates, c/h update, outputs, and the new h
+//            as bf16 planes; then one thread fences and raises the CTA's stamp.
+// Every wait (stamps, mbarriers) is bounded; on expiry the CTA records a timeout status and all roles fall
+// through to the common exit where tensor memory is released.  No TMA multicast is used.
+#include "common.cuh"
+
+#include <cuda.h>
+#include <cstdio>
+#include <cstring>
+
+namespace lstm {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr long long kWaitTicks = 4000000000ll;  // clock64 ticks an mbarrier wait may last (about two seconds)
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; false when it gave up or another role did.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    long long t_start = 0;
+    for (long long it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255) == 255) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t_start == 0) t_start = now;
+            if (now - t_start > kWaitTicks) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// K-major operand tile, 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u32(unsigned *p, unsigned v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_volatile_s32(const int *p)
+{
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+
+__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
+__device__ __forceinline__ float tanh_fast(float z)
+{
+    const float t = __expf(-2.0f * fabsf(z));
+    return copysignf(__fdividef(1.0f - t, 1.0f + t), z);
+}
+__device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
+{
+    const int base = H / nc, rem = H % nc;
+    n = base + (c < rem ? 1 : 0);
+    u0 = c * base + (c < rem ? c : rem);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h, const RecurTcArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ __align__(8) unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar, w_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int H = a.H, B = a.B, T = a.T, D = a.D, N = a.N, S = a.stages, RA = a.RA, nkb = a.nkb;
+    const int d = blockIdx.x / a.ncta_dir;
+    const int cta = blockIdx.x - d * a.ncta_dir;
+    int u0, nu;
+    unit_range(H, a.ncta_dir, cta, u0, nu);
+    const int upc = (H + a.ncta_dir - 1) / a.ncta_dir;
+
+    // shared-memory carve-up (tiles need 1024-byte alignment): weight tiles, operand ring, then scratch
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_tiles = base;                                          // [nkb][RA rows][128 B]
+    const uint32_t ring = a_tiles + (uint32_t)nkb * RA * 128;               // [S][N rows][128 B]
+    unsigned char *gen = smem_raw + (ring + (uint32_t)S * N * 128 - smem_u32(smem_raw));
+    float *zs = reinterpret_cast<float *>(gen);                             // [4*upc][B] gate pre-activations (h part)
+    float *c_s = zs + 4 * upc * B;                                          // [upc][B]
+
+    if (tid == 0) {
+        abort_s = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        mbar_init(smem_u32(&accum_bar), 1);
+        mbar_init(smem_u32(&w_bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    for (int i = tid; i < nu * B; i += kThreads) {
+        const int u = i / B, b = i - u * B;
+        c_s[u * B + b] = a.c0 ? a.c0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_s;
+    volatile int *abort_flag = &abort_s;
+
+    __nv_bfloat16 *hbuf_d = a.hbuf + (size_t)d * 2 * 64 * a.ldh;            // [parity][64 rows][ldh]
+    unsigned *flags_d = a.flags + (size_t)d * a.ncta_dir;
+
+    if (warp == 0) {
+        // ================= stamps and TMA =================
+        if (lane == 0) {
+            // the CTA's weight tiles, once
+            mbar_expect_tx(smem_u32(&w_bar), (uint32_t)nkb * RA * 128);
+            for (int kb = 0; kb < nkb; ++kb)
+                tma_load_2d(a_tiles + (uint32_t)kb * RA * 128, &tmap_w, smem_u32(&w_bar), kb * 64, (d * a.ncta_dir + cta) * RA);
+        }
+        long long i_kb = 0;
+        for (int s = 0; s < T && !*abort_flag; ++s) {
+            // every producer's stamp of the previous step (the prologue publishes h0 with stamp_base)
+            const unsigned want = a.stamp_base + (unsigned)s;
+            long long t_start = 0;
+            int rounds = 0;
+            while (true) {
+                bool ok = true;
+                for (int i = lane; i < a.ncta_dir; i += 32) ok &= (int)(ld_acquire_u32(flags_d + i) - want) >= 0;
+                if (__all_sync(0xffffffffu, ok)) break;
+                if ((++rounds & 15) == 0) {
+                    const long long now = clock64();
+                    if (t_start == 0) t_start = now;
+                    if (now - t_start > a.spin_limit || ld_volatile_s32(a.status) != kStatusOk || *abort_flag) {
+                        *abort_flag = 1;
+                        break;
+                    }
+                }
+            }
+            if (*abort_flag) break;
+            if (lane == 0) {
+                asm volatile("fence.proxy.async;" ::: "memory");       // the planes were written with ordinary stores
+                const int row0 = (d * 2 + ((s + 1) & 1)) * 64;          // planes of step s-1 live in parity (s-1)&1
+                for (int kb = 0; kb < nkb; ++kb, ++i_kb) {
+                    const int st = (int)(i_kb % S);
+                    const uint32_t ph = (uint32_t)(i_kb / S) & 1u;
+                    if (!mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abort_flag)) break;
+                    mbar_expect_tx(smem_u32(&full_bar[st]), (uint32_t)N * 128);
+                    tma_load_2d(ring + (uint32_t)st * N * 128, &tmap_h, smem_u32(&full_bar[st]), kb * 64, row0);
+                }
+            }
+            __syncwarp();
+        }
+    } else if (warp == 1) {
+        // ================= MMA issue =================
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            bool ok = mbar_wait(smem_u32(&w_bar), 0u, abort_flag);
+            long long i_kb = 0;
+            for (int s = 0; s < T && ok; ++s) {
+                for (int kb = 0; kb < nkb && ok; ++kb, ++i_kb) {
+                    const int st = (int)(i_kb % S);
+                    const uint32_t ph = (uint32_t)(i_kb / S) & 1u;
+                    ok = mbar_wait(smem_u32(&full_bar[st]), ph, abort_flag);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t at = a_tiles + (uint32_t)kb * RA * 128;
+                    const uint32_t bt = ring + (uint32_t)st * N * 128;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16(tmem_base, umma_desc_sw128(at + k * 32), umma_desc_sw128(bt + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(&empty_bar[st]));
+                }
+                if (ok) umma_commit(smem_u32(&accum_bar));
+            }
+        }
+    } else {
+        // ================= accumulator read-back and the cell =================
+        const int ftid = tid - 64;                       // 0..127
+        const int lq = warp & 3;                         // TMEM lane quadrant this warp may read
+        // the planes of h0 (stamp_base): this CTA's units
+        for (int p = ftid; p < nu * B; p += 128) {
+            const int u = p / B, b = p - u * B;
+            const float v = a.h0 ? a.h0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            __nv_bfloat16 *row = hbuf_d + ((size_t)1 * 64 + 2 * b) * a.ldh + u0 + u;     // step -1 -> parity 1
+            row[0] = hi;
+            row[a.ldh] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        }
+        bar_sync(1, 128);
+        if (ftid == 0 && (int)blockIdx.x != a.withhold_cta) {
+            __threadfence();
+            st_relaxed_u32(flags_d + cta, a.stamp_base);
+        }
+        for (int s = 0; s < T; ++s) {
+            const int t = d ? (T - 1 - s) : s;
+            if (!mbar_wait(smem_u32(&accum_bar), (uint32_t)s & 1u, abort_flag)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int row = lq * 32 + lane;              // accumulator row = 4 * unit + gate
+            if (lq * 32 < 4 * nu) {
+                for (int c0 = 0; c0 < 2 * B; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (row < 4 * nu) {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 2) {
+                            const int b = (c0 + i) >> 1;
+                            if (b < B) zs[row * B + b] = __uint_as_float(v[i]) + __uint_as_float(v[i + 1]);
+                        }
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            bar_sync(1, 128);
+            __nv_bfloat16 *hp = hbuf_d + (size_t)(s & 1) * 64 * a.ldh;
+            for (int p = ftid; p < nu * B; p += 128) {
+                const int u = p / B, b = p - u * B, j = u0 + u;
+                float4 gsum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)j * 4);
+                for (int sp = 0; sp < a.nsplit; ++sp) {
+                    const float4 g4 = __ldg(gp + (size_t)sp * (a.g_split_stride / 4));
+                    gsum.x += g4.x; gsum.y += g4.y; gsum.z += g4.z; gsum.w += g4.w;
+                }
+                const float gi = sigmoid_fast(zs[(4 * u + 0) * B + b] + gsum.x);
+                const float gf = sigmoid_fast(zs[(4 * u + 1) * B + b] + gsum.y);
+                const float gg = tanh_fast(zs[(4 * u + 2) * B + b] + gsum.z);
+                const float go = sigmoid_fast(zs[(4 * u + 3) * B + b] + gsum.w);
+                const float cn = fmaf(gf, c_s[u * B + b], gi * gg);
+                const float hn = go * tanh_fast(cn);
+                c_s[u * B + b] = cn;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(hn - __bfloat162float(hi));
+                hp[(size_t)(2 * b) * a.ldh + j] = hi;
+                hp[(size_t)(2 * b + 1) * a.ldh + j] = lo;
+                a.y[((size_t)t * B + b) * D * H + (size_t)d * H + j] = hn;
+                if (a.xb_next) {
+                    const size_t xi = ((size_t)t * B + b) * a.xb_ld + (size_t)d * H + j;
+                    a.xb_next[xi] = hi;
+                    a.xb_next[a.xb_plane + xi] = lo;
+                }
+                if (s == T - 1) {
+                    if (a.hT) a.hT[((size_t)d * B + b) * H + j] = hn;
+                    if (a.cT) a.cT[((size_t)d * B + b) * H + j] = cn;
+                }
+            }
+            bar_sync(1, 128);
+            if (ftid == 0 && (int)blockIdx.x != a.withhold_cta) {
+                __threadfence();
+                st_relaxed_u32(flags_d + cta, a.stamp_base + (unsigned)s + 1u);
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+    }
+    if (tid == 0 && abort_s) atomicExch(a.status, kStatusTimeout);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+// rows x cols bf16 matrix, row stride ld elements; box = 64 columns x box_rows, 128-byte swizzle, zero fill
+bool encode_2d(void *map, const void *base, long long rows, int cols, int ld, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(reinterpret_cast<CUtensorMap *>(map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+
+size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int upc, int B)
+{
+    // the last weight tile is read as 128 rows: at least (128 - RA) * 128 bytes must follow it
+    const size_t after = (size_t)stages * N * 128 + (size_t)(4 * upc * B + upc * B) * 4 + 16;
+    const size_t need = (size_t)(128 - RA) * 128;
+    return 1024 + (size_t)nkb * RA * 128 + (after > need ? after : need);
+}
+
+bool recur_tc_encode_weights(void *map, const void *w, long long rows, int ld, int RA)
+{
+    return encode_2d(map, w, rows, ld, ld, RA);
+}
+bool recur_tc_encode_planes(void *map, const void *hbuf, int D, int H, int ldh, int N)
+{
+    return encode_2d(map, hbuf, (long long)D * 2 * 64, H, ldh, N);
+}
+
+cudaError_t recur_tc_prepare(int max_smem)
+{
+    return cudaFuncSetAttribute(recur_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+}
+
+cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurTcArgs &a, size_t smem, cudaStream_t st)
+{
+    CUtensorMap mw, mh;
+    memcpy(&mw, tmap_w, sizeof mw);
+    memcpy(&mh, tmap_h, sizeof mh);
+    RecurTcArgs copy = a;
+    void *params[] = {&mw, &mh, &copy};
+    return cudaLaunchCooperativeKernel((const void *)recur_tc_kernel, dim3(a.ncta_dir * a.D), dim3(kThreads), params, smem, st);
+}
+
+}  // namespace lstm
