@@ -411,7 +411,8 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
         const int RA = round_up(4 * h->upc, 8), nkb = (H + 63) / 64;
         if (h->use_mma && max_B > 4 && RA <= 128 && !(env && strcmp(env, "mma") == 0)) {
             const int B = std::min(max_B, 32), N = round_up(2 * B, 16);
-            if (recur_tc_smem_bytes(RA, nkb, N, std::min(8, nkb), h->upc, B) <= (size_t)h->smem_optin - 256) {
+            int kbs = 0, stages = 0;
+            if (h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - 256, &kbs, &stages)) {
                 h->use_tcb = true; h->tcb_RA = RA; h->tcb_nkb = nkb; h->tcb_ld = nkb * 64; h->tcb_ldh = round_up(H, 8);
             }
         }
@@ -934,7 +935,9 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             RecurTcArgs m;
             memset(&m, 0, sizeof m);
             m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
-            m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16); m.stages = std::min(8, h->tcb_nkb);
+            m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16);
+            if (!recur_tc_plan(m.RA, m.nkb, m.N, h->upc, B, (size_t)h->smem_optin - 256, &m.kbs, &m.stages))
+                return fail(h, LSTM_ERR_INVALID, "batched recurrence does not fit shared memory at batch %d", B);
             m.tmem_cols = m.N <= 32 ? 32 : 64;
             m.ldh = h->tcb_ldh;
             m.stamp_base = h->stamp_next;
@@ -957,7 +960,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
                     return fail(h, LSTM_ERR_CUDA, "tensor map of the h planes could not be encoded");
                 h->tcb_mapN = m.N;
             }
-            const size_t smem = recur_tc_smem_bytes(m.RA, m.nkb, m.N, m.stages, h->upc, B);
+            const size_t smem = recur_tc_smem_bytes(m.RA, m.nkb, m.N, m.stages, m.kbs, h->upc, B);
             if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
             e = launch_recur_tc(ly.tmap_wtc, h->tmap_planes, m, smem, st);
             ++h->last_launches;

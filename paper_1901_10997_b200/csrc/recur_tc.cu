@@ -32,6 +32,9 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
+constexpr int kFlagLoads = 5;                   // stamps one lane polls: up to 160 CTAs per direction
+constexpr int kPre = 2;                         // (unit, batch row) items per thread whose projection terms are prefetched
+constexpr int kMaxSplit = 4;                    // split-K partial sums of the projection
 constexpr long long kWaitTicks = 4000000000ll;  // clock64 ticks an mbarrier wait may last (about two seconds)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -112,6 +115,18 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_nc_f4(const float4 *p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
 __device__ __forceinline__ void st_relaxed_u32(unsigned *p, unsigned v)
 {
     asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -143,10 +158,10 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ __align__(8) unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar, w_bar;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s;
+    __shared__ int abort_s, pub_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int H = a.H, B = a.B, T = a.T, D = a.D, N = a.N, S = a.stages, RA = a.RA, nkb = a.nkb;
+    const int H = a.H, B = a.B, T = a.T, D = a.D, N = a.N, S = a.stages, RA = a.RA, nkb = a.nkb, kbs = a.kbs;
     const int d = blockIdx.x / a.ncta_dir;
     const int cta = blockIdx.x - d * a.ncta_dir;
     int u0, nu;
@@ -156,13 +171,15 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     // shared-memory carve-up (tiles need 1024-byte alignment): weight tiles, operand ring, then scratch
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_tiles = base;                                          // [nkb][RA rows][128 B]
-    const uint32_t ring = a_tiles + (uint32_t)nkb * RA * 128;               // [S][N rows][128 B]
-    unsigned char *gen = smem_raw + (ring + (uint32_t)S * N * 128 - smem_u32(smem_raw));
-    float *zs = reinterpret_cast<float *>(gen);                             // [4*upc][B] gate pre-activations (h part)
-    float *c_s = zs + 4 * upc * B;                                          // [upc][B]
+    const uint32_t ring = a_tiles + (uint32_t)nkb * RA * 128;               // [S][kbs][N rows][128 B]
+    unsigned char *gen = smem_raw + (ring + (uint32_t)(S * kbs * N) * 128 - smem_u32(smem_raw));
+    float *zs = reinterpret_cast<float *>(gen);                             // [B][4*upc] gate pre-activations (h part)
+    const int zld = 4 * upc;
+    float *c_s = zs + zld * B;                                              // [B][units of this CTA]
 
     if (tid == 0) {
         abort_s = 0;
+        pub_s = 0;
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
         mbar_init(smem_u32(&accum_bar), 1);
         mbar_init(smem_u32(&w_bar), 1);
@@ -175,78 +192,114 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     for (int i = tid; i < nu * B; i += kThreads) {
-        const int u = i / B, b = i - u * B;
-        c_s[u * B + b] = a.c0 ? a.c0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
+        const int b = i / nu, u = i - b * nu;
+        c_s[i] = a.c0 ? a.c0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_s;
     volatile int *abort_flag = &abort_s;
+    volatile int *pub = &pub_s;                 // steps this CTA has published (h0 counts as one)
 
     __nv_bfloat16 *hbuf_d = a.hbuf + (size_t)d * 2 * 64 * a.ldh;            // [parity][64 rows][ldh]
     unsigned *flags_d = a.flags + (size_t)d * a.ncta_dir;
 
     if (warp == 0) {
         // ================= stamps and TMA =================
-        if (lane == 0) {
-            // the CTA's weight tiles, once
-            mbar_expect_tx(smem_u32(&w_bar), (uint32_t)nkb * RA * 128);
-            for (int kb = 0; kb < nkb; ++kb)
-                tma_load_2d(a_tiles + (uint32_t)kb * RA * 128, &tmap_w, smem_u32(&w_bar), kb * 64, (d * a.ncta_dir + cta) * RA);
-        }
-        long long i_kb = 0;
-        for (int s = 0; s < T && !*abort_flag; ++s) {
-            // every producer's stamp of the previous step (the prologue publishes h0 with stamp_base)
+        // the CTA's weight tiles, once (one lane per tile)
+        if (lane == 0) mbar_expect_tx(smem_u32(&w_bar), (uint32_t)nkb * RA * 128);
+        __syncwarp();
+        for (int kb = lane; kb < nkb; kb += 32)
+            tma_load_2d(a_tiles + (uint32_t)kb * RA * 128, &tmap_w, smem_u32(&w_bar), kb * 64, (d * a.ncta_dir + cta) * RA);
+        // ring position as a stage index and a phase bit (a 64-bit divide per stage would cost the issuing
+        // thread more than the copies it issues)
+        int st = 0;
+        uint32_t ph = 0;
+        bool live = true;
+        for (int s = 0; s < T && live; ++s) {
+            // Do not poll before this CTA has published its own part of the previous step: loads that spin
+            // ahead of the data queue up in front of the SM's own stores and delay every consumer.
+            if (lane == 0) {
+                long long t_start = 0;
+                for (int it = 0; *pub < s + 1; ++it) {
+                    if ((it & 63) == 63) {
+                        const long long now = clock64();
+                        if (t_start == 0) t_start = now;
+                        if (now - t_start > a.spin_limit || *abort_flag) { *abort_flag = 1; break; }
+                    }
+                }
+            }
+            __syncwarp();
+            // every producer's stamp of the previous step (the prologue publishes h0 with stamp_base): relaxed
+            // loads, all in flight together, and one fence once they all show the stamp
             const unsigned want = a.stamp_base + (unsigned)s;
             long long t_start = 0;
             int rounds = 0;
+            bool aborted = false;
             while (true) {
+                unsigned v[kFlagLoads];
+#pragma unroll
+                for (int k = 0; k < kFlagLoads; ++k) {
+                    const int i = lane + 32 * k;
+                    v[k] = i < a.ncta_dir ? ld_relaxed_u32(flags_d + i) : want;
+                }
                 bool ok = true;
-                for (int i = lane; i < a.ncta_dir; i += 32) ok &= (int)(ld_acquire_u32(flags_d + i) - want) >= 0;
+#pragma unroll
+                for (int k = 0; k < kFlagLoads; ++k) ok &= (int)(v[k] - want) >= 0;
+                // both votes are taken by all lanes every round, so the warp leaves the loop as one
+                if (__any_sync(0xffffffffu, *abort_flag != 0)) { aborted = true; break; }
                 if (__all_sync(0xffffffffu, ok)) break;
                 if ((++rounds & 15) == 0) {
                     const long long now = clock64();
                     if (t_start == 0) t_start = now;
-                    if (now - t_start > a.spin_limit || ld_volatile_s32(a.status) != kStatusOk || *abort_flag) {
-                        *abort_flag = 1;
-                        break;
-                    }
+                    if (now - t_start > a.spin_limit || ld_volatile_s32(a.status) != kStatusOk) *abort_flag = 1;
                 }
             }
-            if (*abort_flag) break;
-            if (lane == 0) {
-                asm volatile("fence.proxy.async;" ::: "memory");       // the planes were written with ordinary stores
-                const int row0 = (d * 2 + ((s + 1) & 1)) * 64;          // planes of step s-1 live in parity (s-1)&1
-                for (int kb = 0; kb < nkb; ++kb, ++i_kb) {
-                    const int st = (int)(i_kb % S);
-                    const uint32_t ph = (uint32_t)(i_kb / S) & 1u;
-                    if (!mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abort_flag)) break;
-                    mbar_expect_tx(smem_u32(&full_bar[st]), (uint32_t)N * 128);
-                    tma_load_2d(ring + (uint32_t)st * N * 128, &tmap_h, smem_u32(&full_bar[st]), kb * 64, row0);
+            if (aborted) break;
+            __threadfence();                                        // acquire: the planes behind the stamps
+            asm volatile("fence.proxy.async;" ::: "memory");       // they were written with ordinary stores
+            const int row0 = (d * 2 + ((s + 1) & 1)) * 64;          // planes of step s-1 live in parity (s-1)&1
+            for (int g0 = 0; g0 < nkb; g0 += kbs) {
+                const int nblk = min(kbs, nkb - g0);
+                int ok = 1;
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abort_flag) ? 1 : 0;
+                    if (ok) mbar_expect_tx(smem_u32(&full_bar[st]), (uint32_t)(nblk * N) * 128);
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { live = false; break; }
+                // one lane per K block of the stage: issuing a tensor copy occupies a thread for a while
+                if (lane < nblk)
+                    tma_load_2d(ring + (uint32_t)((st * kbs + lane) * N) * 128, &tmap_h, smem_u32(&full_bar[st]), (g0 + lane) * 64, row0);
+                if (++st == S) { st = 0; ph ^= 1u; }
             }
-            __syncwarp();
         }
     } else if (warp == 1) {
         // ================= MMA issue =================
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
             bool ok = mbar_wait(smem_u32(&w_bar), 0u, abort_flag);
-            long long i_kb = 0;
+            // descriptors differ only in their start-address field (units of 16 bytes): build one of each and add
+            const uint64_t adesc0 = umma_desc_sw128(a_tiles), bdesc0 = umma_desc_sw128(ring);
+            const uint32_t a_step = (uint32_t)(RA * 128) >> 4, b_step = (uint32_t)(N * 128) >> 4;
+            int st = 0;
+            uint32_t ph = 0;
             for (int s = 0; s < T && ok; ++s) {
-                for (int kb = 0; kb < nkb && ok; ++kb, ++i_kb) {
-                    const int st = (int)(i_kb % S);
-                    const uint32_t ph = (uint32_t)(i_kb / S) & 1u;
+                uint64_t adesc = adesc0;
+                for (int g0 = 0; g0 < nkb; g0 += kbs) {
+                    const int nblk = min(kbs, nkb - g0);
                     ok = mbar_wait(smem_u32(&full_bar[st]), ph, abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t at = a_tiles + (uint32_t)kb * RA * 128;
-                    const uint32_t bt = ring + (uint32_t)st * N * 128;
+                    uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)(st * kbs) * b_step);
+                    for (int l = 0; l < nblk; ++l, adesc += a_step, bdesc += b_step) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem_base, umma_desc_sw128(at + k * 32), umma_desc_sw128(bt + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (g0 + l > 0 || k > 0) ? 1u : 0u);
+                    }
                     umma_commit(smem_u32(&empty_bar[st]));
+                    if (++st == S) { st = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(smem_u32(&accum_bar));
             }
@@ -255,9 +308,10 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         // ================= accumulator read-back and the cell =================
         const int ftid = tid - 64;                       // 0..127
         const int lq = warp & 3;                         // TMEM lane quadrant this warp may read
+        const int nuB = nu * B;
         // the planes of h0 (stamp_base): this CTA's units
-        for (int p = ftid; p < nu * B; p += 128) {
-            const int u = p / B, b = p - u * B;
+        for (int p = ftid; p < nuB; p += 128) {
+            const int b = p / nu, u = p - b * nu;
             const float v = a.h0 ? a.h0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
             __nv_bfloat16 *row = hbuf_d + ((size_t)1 * 64 + 2 * b) * a.ldh + u0 + u;     // step -1 -> parity 1
@@ -265,12 +319,29 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             row[a.ldh] = __float2bfloat16_rn(v - __bfloat162float(hi));
         }
         bar_sync(1, 128);
-        if (ftid == 0 && (int)blockIdx.x != a.withhold_cta) {
-            __threadfence();
-            st_relaxed_u32(flags_d + cta, a.stamp_base);
+        if (ftid == 0) {
+            if ((int)blockIdx.x != a.withhold_cta) {
+                __threadfence();
+                st_relaxed_u32(flags_d + cta, a.stamp_base);
+            }
+            *pub = 1;
         }
+        const size_t gs4 = (size_t)(a.g_split_stride / 4);
         for (int s = 0; s < T; ++s) {
             const int t = d ? (T - 1 - s) : s;
+            // projection terms of the first items: requested before the wait, they do not depend on h
+            float4 gpre[kPre][kMaxSplit];
+#pragma unroll
+            for (int i = 0; i < kPre; ++i) {
+                const int p = ftid + 128 * i;
+                if (p < nuB) {
+                    const int b = p / nu, j = u0 + p - b * nu;
+                    const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)j * 4);
+#pragma unroll
+                    for (int sp = 0; sp < kMaxSplit; ++sp)
+                        if (sp < a.nsplit) gpre[i][sp] = ld_nc_f4(gp + (size_t)sp * gs4);
+                }
+            }
             if (!mbar_wait(smem_u32(&accum_bar), (uint32_t)s & 1u, abort_flag)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int row = lq * 32 + lane;              // accumulator row = 4 * unit + gate
@@ -281,9 +352,9 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     if (row < 4 * nu) {
 #pragma unroll
-                        for (int i = 0; i < 16; i += 2) {
-                            const int b = (c0 + i) >> 1;
-                            if (b < B) zs[row * B + b] = __uint_as_float(v[i]) + __uint_as_float(v[i + 1]);
+                        for (int i = 0; i < 8; ++i) {
+                            const int b = (c0 >> 1) + i;
+                            if (b < B) zs[b * zld + row] = __uint_as_float(v[2 * i]) + __uint_as_float(v[2 * i + 1]);
                         }
                     }
                 }
@@ -291,21 +362,34 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             bar_sync(1, 128);
             __nv_bfloat16 *hp = hbuf_d + (size_t)(s & 1) * 64 * a.ldh;
-            for (int p = ftid; p < nu * B; p += 128) {
-                const int u = p / B, b = p - u * B, j = u0 + u;
+            for (int i = 0; ftid + 128 * i < nuB; ++i) {
+                const int p = ftid + 128 * i;
+                const int b = p / nu, u = p - b * nu, j = u0 + u;       // consecutive threads, consecutive units
                 float4 gsum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)j * 4);
-                for (int sp = 0; sp < a.nsplit; ++sp) {
-                    const float4 g4 = __ldg(gp + (size_t)sp * (a.g_split_stride / 4));
-                    gsum.x += g4.x; gsum.y += g4.y; gsum.z += g4.z; gsum.w += g4.w;
+                if (i < kPre) {
+#pragma unroll
+                    for (int ii = 0; ii < kPre; ++ii) {
+                        if (ii == i) {
+#pragma unroll
+                            for (int sp = 0; sp < kMaxSplit; ++sp)
+                                if (sp < a.nsplit) { gsum.x += gpre[ii][sp].x; gsum.y += gpre[ii][sp].y; gsum.z += gpre[ii][sp].z; gsum.w += gpre[ii][sp].w; }
+                        }
+                    }
+                } else {
+                    const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)j * 4);
+                    for (int sp = 0; sp < a.nsplit; ++sp) {
+                        const float4 g4 = __ldg(gp + (size_t)sp * gs4);
+                        gsum.x += g4.x; gsum.y += g4.y; gsum.z += g4.z; gsum.w += g4.w;
+                    }
                 }
-                const float gi = sigmoid_fast(zs[(4 * u + 0) * B + b] + gsum.x);
-                const float gf = sigmoid_fast(zs[(4 * u + 1) * B + b] + gsum.y);
-                const float gg = tanh_fast(zs[(4 * u + 2) * B + b] + gsum.z);
-                const float go = sigmoid_fast(zs[(4 * u + 3) * B + b] + gsum.w);
-                const float cn = fmaf(gf, c_s[u * B + b], gi * gg);
+                const float4 z4 = *reinterpret_cast<const float4 *>(zs + b * zld + 4 * u);
+                const float gi = sigmoid_fast(z4.x + gsum.x);
+                const float gf = sigmoid_fast(z4.y + gsum.y);
+                const float gg = tanh_fast(z4.z + gsum.z);
+                const float go = sigmoid_fast(z4.w + gsum.w);
+                const float cn = fmaf(gf, c_s[p], gi * gg);
                 const float hn = go * tanh_fast(cn);
-                c_s[u * B + b] = cn;
+                c_s[p] = cn;
                 const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
                 const __nv_bfloat16 lo = __float2bfloat16_rn(hn - __bfloat162float(hi));
                 hp[(size_t)(2 * b) * a.ldh + j] = hi;
@@ -322,9 +406,12 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                 }
             }
             bar_sync(1, 128);
-            if (ftid == 0 && (int)blockIdx.x != a.withhold_cta) {
-                __threadfence();
-                st_relaxed_u32(flags_d + cta, a.stamp_base + (unsigned)s + 1u);
+            if (ftid == 0) {
+                if ((int)blockIdx.x != a.withhold_cta) {
+                    __threadfence();
+                    st_relaxed_u32(flags_d + cta, a.stamp_base + (unsigned)s + 1u);
+                }
+                *pub = s + 2;
             }
         }
     }
@@ -370,12 +457,29 @@ bool encode_2d(void *map, const void *base, long long rows, int cols, int ld, in
 
 static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
 
-size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int upc, int B)
+size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc, int B)
 {
     // the last weight tile is read as 128 rows: at least (128 - RA) * 128 bytes must follow it
-    const size_t after = (size_t)stages * N * 128 + (size_t)(4 * upc * B + upc * B) * 4 + 16;
+    const size_t after = (size_t)stages * kbs * N * 128 + (size_t)(4 * upc * B + upc * B) * 4 + 16;
     const size_t need = (size_t)(128 - RA) * 128;
     return 1024 + (size_t)nkb * RA * 128 + (after > need ? after : need);
+}
+
+// Ring shape for one launch: stages of up to four K blocks (one mbarrier round trip per stage instead of per
+// block), as many stages as fit, at least two unless one stage holds the whole operand.
+bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int *kbs_out, int *stages_out)
+{
+    for (int kbs = nkb < 4 ? nkb : 4; kbs >= 1; --kbs) {
+        const int groups = (nkb + kbs - 1) / kbs;
+        for (int st = groups < kMaxStages ? groups : kMaxStages; st >= (groups > 1 ? 2 : 1); --st) {
+            if (recur_tc_smem_bytes(RA, nkb, N, st, kbs, upc, B) <= max_smem) {
+                *kbs_out = kbs;
+                *stages_out = st;
+                return true;
+            }
+        }
+    }
+    return false;
 }
 
 bool recur_tc_encode_weights(void *map, const void *w, long long rows, int ld, int RA)
