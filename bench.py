@@ -356,7 +356,8 @@ def run_gpu(args):
         achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
         info = model.info()
         kernel_name, kernel_src = (("hlstm_mma_kernel", "hlstm_mma.cu") if mode == "hlstm" else
-                                   ("recur_mma_kernel", "recur_mma.cu") if info.get("recur_register_resident")
+                                   ("recur_tc_kernel", "recur_tc.cu") if info.get("recur_batched_tensor_core")
+                                   else ("recur_mma_kernel", "recur_mma.cu") if info.get("recur_register_resident")
                                    else ("recur_kernel", "recur.cu"))
         traffic = measured_traffic(kernel_name, args.workload, kernel_src)
         line = {

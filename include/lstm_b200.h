@@ -197,7 +197,9 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
  * [6] split-K factor of the input projection at max_T*max_B, [7] 1 if the projection uses the tensor-core
  * (tcgen05) kernel, [8] kernels launched by the most recent lstm_forward (before the first call: the count expected),
  * [9] 1 if the recurrence keeps its weights in registers (bf16 dense), 0 for the shared-memory kernel,
- * [10] 16-column weight tiles per warp held in registers, [11] per warp held in shared memory.
+ * [10] 16-column weight tiles per warp held in registers, [11] per warp held in shared memory,
+ * [12] 1 if a call at max_B runs the batched tensor-core (tcgen05) recurrence: bf16 dense LSTM handles use
+ * it for batches of 5 to 32 sequences and the register-resident kernel below that.
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 

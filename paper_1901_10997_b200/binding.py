@@ -144,7 +144,7 @@ def lstm_info(handle):
     n = load_library().lstm_info(handle, out, 16)
     keys = ["sm_count", "ctas_per_dir", "threads", "smem_bytes", "rows_resident", "rows_streamed",
             "proj_splits", "proj_tensor_core", "launches_per_forward", "recur_register_resident",
-            "col_tiles_in_registers", "col_tiles_in_smem"]
+            "col_tiles_in_registers", "col_tiles_in_smem", "recur_batched_tensor_core"]
     return {k: int(out[i]) for i, k in enumerate(keys[:n])}
 
 

@@ -1156,11 +1156,12 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
     }
     const Layer &l0 = h->layers[0];
     const int launches = h->last_launches > 0 ? h->last_launches : h->L * 2 + (h->use_tc ? 1 : 0);
-    const int64_t vals[12] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->threads, (int64_t)shp.smem,
+    const int tcb_at_max = (h->use_tcb && !h->Hh && h->max_B > 4 && h->max_B <= 32) ? 1 : 0;
+    const int64_t vals[13] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->threads, (int64_t)shp.smem,
                               rows_res, rows_str, (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches,
-                              h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0};
-    for (int i = 0; i < n && i < 12; ++i) out[i] = vals[i];
-    return 12;
+                              h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0, tcb_at_max};
+    for (int i = 0; i < n && i < 13; ++i) out[i] = vals[i];
+    return 13;
 }
 
 }  // extern "C"

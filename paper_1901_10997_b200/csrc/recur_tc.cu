@@ -11,14 +11,16 @@
 // shared memory as 128-byte-swizzled K-major tiles (one per 64 columns) and stays there.  h travels
 // between CTAs through global memory as the tensor cores want it: two bf16 planes per batch row (row 2b =
 // hi, row 2b+1 = lo, so products keep about 16 mantissa bits), K-major.  Per step:
-//   warp 0   polls one stamp per producer CTA (acquire loads, bounded), then streams the [2B x H] operand
-//            into a ring of shared-memory stages with TMA (64 columns per stage, zero fill at the tail);
+//   warp 0   waits until its own CTA has published the previous step, polls one stamp per producer CTA
+//            (relaxed loads, all in flight together, one fence after the last; bounded), then streams the
+//            [2B x H] operand into a ring of shared-memory stages with TMA (up to four 64-column blocks per
+//            stage, one issuing lane per block, zero fill at the tail);
 //   warp 1   issues M = 128, N = 2B (rounded up to 16), K = 16 tcgen05.mma instructions into one TMEM
 //            accumulator; the weight tile has only 4*units (<= 128) real rows: the rows beyond read whatever
 //            follows in shared memory and produce accumulator rows nobody reads;
-//   warps 2-5 read the accumulator rows of the CTA's units back (tcgen05.ld), add hi and lo columns, and
-//            finish the (unit, batch row) pairs: projection term, gates, c/h update, outputs, and the new h
-//            as bf16 planes; then one thread fences and raises the CTA's stamp.
+//   warps 2-5 request their projection terms, then read the accumulator rows of the CTA's units back
+//            (tcgen05.ld), add hi and lo columns, and finish the (unit, batch row) pairs: gates, c/h update,
+//            outputs, and the new h as bf16 planes; then one thread fences and raises the CTA's stamp.
 // Every wait (stamps, mbarriers) is bounded; on expiry the CTA records a timeout status and all roles fall
 // through to the common exit where tensor memory is released.  No TMA multicast is used.
 #include "common.cuh"
