@@ -396,16 +396,13 @@ def run_gpu(args):
 
 
 def lhp_analysis(hs, lat, eps):
-    """Latency-hysteresis points (paper, Section 3): scanning from the largest size down, a size is an
-    LHP if no larger size is at most (1+eps) times as slow; every other size is dominated (a larger
-    model runs at least as fast).  Redundancy = (1 - #LHP / #points) * 100 %."""
-    lhps, best = [], float("inf")
-    for h, t in sorted(zip(hs, lat), reverse=True):
-        if t * (1 + eps) < best:
-            lhps.append(h)
-        best = min(best, t)
-    lhps.sort()
-    return lhps, (1 - len(lhps) / len(hs)) * 100.0
+    """Latency-hysteresis points of a measured curve (paper, Section 3) through the library's own
+    helper: returns (sorted LHP sizes, redundancy in percent = (1 - #LHP / #points) * 100)."""
+    import paper_1901_10997_b200 as pkg
+    rc, flags, count = pkg.lstm_lhp_points(list(hs), list(lat), eps)
+    if rc != pkg.LSTM_OK:
+        raise RuntimeError(f"lstm_lhp_points failed with code {rc}")
+    return sorted(h for h, f in zip(hs, flags) if f), (1 - count / len(hs)) * 100.0
 
 
 def run_sweep(args):

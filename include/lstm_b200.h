@@ -204,6 +204,36 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 
 /*
+ * Latency hysteresis (Section 3): on a measured latency-versus-size curve a size is a latency hysteresis
+ * point (LHP) when no LARGER size runs within (1 + eps) of its latency; every other size is dominated
+ * (a larger model is at least as fast) and the share of dominated sizes is the paper's architecture-space
+ * redundancy.  Host arrays, no GPU work:
+ *   sizes[n] distinct positive sizes in any order, latency[n] > 0 in any one unit, eps >= 0 the relative
+ *   timing noise below which two latencies count as equal.
+ * lstm_lhp_points writes is_lhp[i] in {0,1} and, if count is not NULL, the number of LHPs.
+ * lstm_nearest_lhp returns in *out_size the smallest LHP >= requested (the size a pruned model is grown
+ * back to, step (c) of Section 5.1); LSTM_ERR_UNSUPPORTED when requested exceeds every measured size.
+ * Both return LSTM_ERR_INVALID for NULL arrays, n <= 0, eps < 0, a non-positive or non-finite latency, or
+ * a repeated size.
+ */
+LSTM_API int lstm_lhp_points(const int *sizes, const double *latency, int n, double eps, int *is_lhp, int *count);
+LSTM_API int lstm_nearest_lhp(const int *sizes, const double *latency, int n, double eps, int requested, int *out_size);
+
+/*
+ * Folds a per-feature affine map on a layer's INPUT into that layer's input weights (Section 5.2 uses
+ * batch normalisation between recurrent layers; with its statistics frozen it is x' = scale * x + shift
+ * per feature, scale = gamma / sqrt(var + epsilon), shift = beta - mean * scale):
+ *     Wx (scale * x + shift) + b  =  (Wx diag(scale)) x + (b + Wx shift)
+ * Host arrays: wx [rows, cols] row-major, b [rows] or NULL (zeros), scale, shift [cols] (either may be
+ * NULL: ones / zeros); writes wx_out [rows, cols] (may be wx itself) and b_out [rows] (may be b itself).
+ * The bias sum is accumulated in double.  Apply it to each (layer, direction) that reads normalised
+ * input, before lstm_create; the pruning mask, if any, applies to the folded matrix unchanged.
+ * Returns LSTM_ERR_INVALID for NULL wx / outputs or non-positive sizes.
+ */
+LSTM_API int lstm_fold_input_affine(const float *wx, const float *b, int rows, int cols, const float *scale,
+                                    const float *shift, float *wx_out, float *b_out);
+
+/*
  * Forward pass without any allocation (the paper has no counterpart: this exists for deployment).
  * For callers that cannot allocate device memory at call time or at all -- a serving loop whose memory
  * pool is fixed at start-up, a host framework whose allocator owns the device, a process that must not

@@ -76,6 +76,13 @@ def load_library():
         lib.lstm_selftest_timeout.argtypes = [vp, ci, ctypes.c_longlong]
         lib.lstm_forward_noalloc.restype = ci
         lib.lstm_forward_noalloc.argtypes = [vp, vp, vp, ci, ci, vp, ci, ci, vp, vp, vp, vp, vp, vp, ctypes.c_char_p, ci]
+        pi, pd, pf = ctypes.POINTER(ci), ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_float)
+        lib.lstm_lhp_points.restype = ci
+        lib.lstm_lhp_points.argtypes = [pi, pd, ci, ctypes.c_double, pi, pi]
+        lib.lstm_nearest_lhp.restype = ci
+        lib.lstm_nearest_lhp.argtypes = [pi, pd, ci, ctypes.c_double, ci, pi]
+        lib.lstm_fold_input_affine.restype = ci
+        lib.lstm_fold_input_affine.argtypes = [pf, pf, ci, ci, pf, pf, pf, pf]
         _lib = lib
     return _lib
 
@@ -146,6 +153,44 @@ def lstm_info(handle):
             "proj_splits", "proj_tensor_core", "launches_per_forward", "recur_register_resident",
             "col_tiles_in_registers", "col_tiles_in_smem", "recur_batched_tensor_core"]
     return {k: int(out[i]) for i, k in enumerate(keys[:n])}
+
+
+def _curve(sizes, latency):
+    n = len(sizes)
+    if n != len(latency):
+        raise ValueError("sizes and latency differ in length")
+    return (ctypes.c_int * n)(*[int(v) for v in sizes]), (ctypes.c_double * n)(*[float(v) for v in latency]), n
+
+
+def lstm_lhp_points(sizes, latency, eps=0.0):
+    """Returns (code, flags, count): flags[i] = 1 where sizes[i] is a latency hysteresis point."""
+    cs, cl, n = _curve(sizes, latency)
+    flags = (ctypes.c_int * max(n, 1))()
+    count = ctypes.c_int(0)
+    rc = load_library().lstm_lhp_points(cs, cl, n, float(eps), flags, ctypes.byref(count))
+    return rc, [int(flags[i]) for i in range(n)], int(count.value)
+
+
+def lstm_nearest_lhp(sizes, latency, requested, eps=0.0):
+    """Returns (code, size): the smallest latency hysteresis point >= requested."""
+    cs, cl, n = _curve(sizes, latency)
+    out = ctypes.c_int(0)
+    rc = load_library().lstm_nearest_lhp(cs, cl, n, float(eps), int(requested), ctypes.byref(out))
+    return rc, int(out.value)
+
+
+def lstm_fold_input_affine(wx, b, scale, shift):
+    """Returns (code, wx_folded, b_folded) as new float32 arrays; b, scale, shift may be None."""
+    import numpy as np
+    wx = np.ascontiguousarray(wx, dtype=np.float32)
+    rows, cols = wx.shape
+    as_f = lambda a, n: None if a is None else np.ascontiguousarray(a, dtype=np.float32).reshape(n)
+    b, scale, shift = as_f(b, rows), as_f(scale, cols), as_f(shift, cols)
+    wx_out, b_out = np.empty_like(wx), np.empty(rows, np.float32)
+    pf = ctypes.POINTER(ctypes.c_float)
+    ptr = lambda a: None if a is None else a.ctypes.data_as(pf)
+    rc = load_library().lstm_fold_input_affine(ptr(wx), ptr(b), rows, cols, ptr(scale), ptr(shift), ptr(wx_out), ptr(b_out))
+    return rc, wx_out, b_out
 
 
 def lstm_forward_noalloc(wx, wh, b, in_dim, hidden, x, T, B, h0, c0, y, hT, cT, stream=0):
