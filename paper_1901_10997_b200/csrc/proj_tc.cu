@@ -150,9 +150,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer
+            int s = 0;
+            uint32_t ph = 0;
             for (int i = 0; i < nkb; ++i) {
-                const int s = i % S;
-                const uint32_t ph = (uint32_t)(i / S) & 1u;
                 if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag)) break;
                 const uint32_t fb = smem_u32(&full_bar[s]);
                 mbar_expect_tx(fb, stage_bytes);
@@ -160,31 +160,32 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 tma_load_2d(sa, &tmap_w, fb, (kb0 + i) * kBK, w_tile * kBM);
                 tma_load_2d(sa + a_bytes, &tmap_x, fb, (kb0 + i) * kBK, x_tile * a.n_tile);
                 tma_load_2d(sa + a_bytes + b_bytes, &tmap_xlo, fb, (kb0 + i) * kBK, x_tile * a.n_tile);
+                if (++s == S) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer
-            // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = n_tile, M = 128
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.n_tile >> 3) << 17) |
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = 128, N = 2 * n_tile: the
+            // hi and the lo activation tiles lie back to back in the stage and form ONE operand of 2 * n_tile
+            // rows (an instruction of this size costs the same whatever N, so one is half the price of two);
+            // accumulator columns [0, n_tile) hold the hi product, [n_tile, 2 n_tile) the lo product
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * a.n_tile) >> 3) << 17) |
                                    ((uint32_t)(kBM >> 4) << 24);
             bool ok = true;
+            int s = 0;
+            uint32_t ph = 0;
             for (int i = 0; i < nkb && ok; ++i) {
-                const int s = i % S;
-                const uint32_t ph = (uint32_t)(i / S) & 1u;
                 ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t sa = tiles + (uint32_t)s * stage_bytes;
+                const uint64_t adesc = umma_desc_sw128(sa), bdesc = umma_desc_sw128(sa + a_bytes);
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k) {
-                    const uint64_t adesc = umma_desc_sw128(sa + k * 32);
-                    const uint64_t bhi = umma_desc_sw128(sa + a_bytes + k * 32);
-                    const uint64_t blo = umma_desc_sw128(sa + a_bytes + b_bytes + k * 32);
-                    umma_bf16(tmem_base, adesc, bhi, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                    umma_bf16(tmem_base, adesc, blo, idesc, 1u);
-                }
+                for (int k = 0; k < kBK / 16; ++k)
+                    umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
                 umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
+                if (++s == S) { s = 0; ph ^= 1u; }
             }
             if (ok) umma_commit(smem_u32(&accum_bar));     // accumulator complete
         }
@@ -198,14 +199,15 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             const float bv = (split == 0 && a.bias && n < a.N) ? a.bias[n] : 0.0f;
             float *gout = a.G + (size_t)split * a.g_split_stride;
             for (int c0 = 0; c0 < a.n_tile; c0 += 16) {
-                uint32_t v[16];
+                uint32_t v[16], vlo[16];
                 tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
+                tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(a.n_tile + c0), vlo);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int m0 = x_tile * a.n_tile + c0;
                 if (n < a.N) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        if (m0 + i < a.M) gout[(size_t)(m0 + i) * a.N + n] = __uint_as_float(v[i]) + bv;
+                        if (m0 + i < a.M) gout[(size_t)(m0 + i) * a.N + n] = __uint_as_float(v[i]) + __uint_as_float(vlo[i]) + bv;
                 }
             }
         }
@@ -308,7 +310,7 @@ cudaError_t launch_proj_tc(const ProjTcPlan &p, const float *bias, float *G, int
     if (stages < 1) stages = 1;
     a.stages = stages;
     int cols = 32;
-    while (cols < p.n_tile) cols <<= 1;
+    while (cols < 2 * p.n_tile) cols <<= 1;      // hi and lo products side by side
     a.tmem_cols = cols;
     a.G = G; a.bias = bias; a.status = status;
     a.g_split_stride = (long long)p.M * p.N;
