@@ -207,13 +207,58 @@ def test_shared_memory_kernel_serves_bf16_dense_when_selected(oracle, monkeypatc
         m.close()
 
 
-@pytest.mark.parametrize("dtype,mode", [("bf16", "dense"), ("fp32", "dense"), ("bf16", "csr")])
-def test_withheld_exchange_words_end_in_a_timeout_status_not_a_hang(oracle, dtype, mode):
-    """One CTA withholds its h values; the waits of the others run out after a millisecond, the call
-    reports LSTM_ERR_TIMEOUT, and the same handle computes correctly again afterwards."""
+# batches of 5..32 sequences on bf16 dense handles run the batched tensor-core recurrence: its edges
+TC_SHAPES = [
+    small("tc_h7_b6", 1, True, 5, 7, 3, 6, "bf16"),                 # one K block, a few rows per CTA, most CTAs with one unit
+    small("tc_h64_b5_t1", 1, False, 20, 64, 1, 5, "bf16"),          # a single step: only the published h0 is consumed
+    small("tc_h129_b32", 1, False, 33, 129, 4, 32, "bf16"),         # the largest batch (N = 64), ragged K tail of one column
+    small("tc_h1000_b17", 2, False, 64, 1000, 3, 17, "bf16", scale=0.05),   # 16 K blocks, four per stage; two layers
+    small("tc_h1600_b9", 1, False, 32, 1600, 2, 9, "bf16", scale=0.03),     # 25 K blocks: the ring is down to a few stages
+    # 14 units per CTA x 32 K blocks do not fit shared memory: the handle keeps the register-resident kernel
+    small("notc_h2000_b9", 1, False, 32, 2000, 2, 9, "bf16", scale=0.03),
+]
+
+
+@pytest.mark.parametrize("w", TC_SHAPES, ids=lambda w: w.name)
+def test_batched_tensor_core_recurrence(oracle, w):
     import torch
     import paper_1901_10997_b200 as pkg
-    w = small("timeout", 1, False, 40, 300, 8, 2, dtype, seed=22)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    m = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype="bf16", max_T=w.T, max_B=w.B)
+    assert m.info()["recur_batched_tensor_core"] == (0 if w.name.startswith("notc") else 1)
+    y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
+    m.check()
+    assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", w.name)
+    # a smaller batch on the same handle goes through the register-resident kernel and must agree too
+    if w.B > 6:
+        nb = 3
+        xs, hs, cs = x[:, :nb].copy(), h0[:, :nb].copy(), c0[:, :nb].copy()
+        y2, h2, c2 = m.forward(torch.from_numpy(xs).cuda(), torch.from_numpy(hs).cuda(), torch.from_numpy(cs).cuda())
+        m.check()
+        assert_close((y2.cpu().numpy(), h2.cpu().numpy(), c2.cpu().numpy()), (ref[0][:, :nb], ref[1][:, :nb], ref[2][:, :nb]), "bf16", w.name + "/b3")
+    m.close()
+
+
+def test_batched_recurrence_chunked_calls_carry_state(oracle):
+    w = small("tc_chunk", 2, True, 24, 150, 9, 8, "bf16", seed=9)
+    weights, x = wl.make(w)
+    # state carried across calls is only defined for one direction per call order; use the forward stack
+    wf = w.with_(bidir=False)
+    weights, x = wl.make(wf)
+    ref = oracle.forward(weights, x, layers=2, bidir=False, hidden=wf.hidden)
+    assert_close(run_gpu(wf, weights, x, chunks=[4, 1, 4]), ref, "bf16", "tc chunked")
+
+
+@pytest.mark.parametrize("dtype,mode,B", [("bf16", "dense", 2), ("fp32", "dense", 2), ("bf16", "csr", 2), ("bf16", "dense", 6)])
+def test_withheld_exchange_words_end_in_a_timeout_status_not_a_hang(oracle, dtype, mode, B):
+    """One CTA withholds its h values (B = 6: its stamp, in the batched kernel); the waits of the others run
+    out after a millisecond, the call reports LSTM_ERR_TIMEOUT, and the same handle computes correctly
+    again afterwards."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = small("timeout", 1, False, 40, 300, 8, B, dtype, seed=22)
     weights, x = wl.make(w)
     ref = oracle.forward(weights, x, layers=1, bidir=False, hidden=w.hidden)
     m = pkg.LSTM(weights, layers=1, in_dim=w.in_dim, hidden=w.hidden, dtype=dtype, exec_mode=mode, max_T=w.T, max_B=w.B)
