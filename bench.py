@@ -406,40 +406,61 @@ def lhp_analysis(hs, lat, eps):
 
 
 def run_sweep(args):
+    """Latency against hidden width with the hysteresis analysis (paper, Section 3).  Shape "cfg3": one
+    layer, input = hidden = H, T = 35, batch 1 (the recurrent stack of Figure 2's kind).  Shape "ds2": the
+    speech-model stack (5 bidirectional layers, 1312 -> H, then 2H -> H, T = 400) at batch 16, the
+    setting of the paper's Figure 3."""
     import torch
     import paper_1901_10997_b200 as pkg
     dev = torch.device("cuda", 0)
     flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
     outdir = ROOT / "gpurun_out"
     outdir.mkdir(exist_ok=True)
-    sizes = wl.config3_sizes() if not args.sweep_sizes else [int(s) for s in args.sweep_sizes.split(",")]
+    ds2 = args.sweep_shape == "ds2"
+    default_sizes = list(range(256, 1536 + 1, 16)) if ds2 else wl.config3_sizes()
+    sizes = default_sizes if not args.sweep_sizes else [int(s) for s in args.sweep_sizes.split(",")]
+    parity_sizes = set(sizes) if not ds2 else {sizes[0], sizes[len(sizes) // 2], sizes[-1]}
     rows = []
     for H in sizes:
-        w = wl.config3(H)
+        w = wl.config5_width(H, 16) if ds2 else wl.config3(H)
         weights, x = wl.make(w)
-        m = pkg.LSTM(weights, layers=1, in_dim=H, hidden=H, dtype="bf16", max_T=w.T, max_B=1)
+        D = 2 if w.bidir else 1
+        m = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=H, bidir=w.bidir, dtype="bf16", max_T=w.T, max_B=w.B)
         xd = torch.from_numpy(x).to(dev)
-        out = (torch.empty((w.T, 1, H), device=dev), torch.empty((1, 1, H), device=dev), torch.empty((1, 1, H), device=dev))
+        out = (torch.empty((w.T, w.B, D * H), device=dev), torch.empty((w.layers * D, w.B, H), device=dev),
+               torch.empty((w.layers * D, w.B, H), device=dev))
         ms = time_steps(lambda: m.forward(xd, out=out), args.steps, max(args.warmup, 3), flush_buf, torch)
         m.check()
         err = None
-        if args.sweep_parity:
+        if args.sweep_parity and H in parity_sizes:
             import oracle
-            ref = oracle.forward(weights, x, layers=1, bidir=False, hidden=H)
-            err = max(wl.rel_err(g.cpu().numpy(), r)[0] for g, r in zip(out, ref))
+            if ds2:
+                # the oracle cannot walk 400 steps x 16 columns at every width: a 24-step call on the same
+                # handle, all 16 columns on the GPU, the first column against the oracle
+                Tp = 24
+                got = m.forward(xd[:Tp].contiguous())
+                m.check()
+                ref = oracle.forward(weights, x[:Tp, :1], layers=w.layers, bidir=True, hidden=H)
+                err = max(wl.rel_err(g[:, :1].cpu().numpy(), r)[0] for g, r in zip(got, ref))
+            else:
+                ref = oracle.forward(weights, x, layers=1, bidir=False, hidden=H)
+                err = max(wl.rel_err(g.cpu().numpy(), r)[0] for g, r in zip(out, ref))
         info = m.info()
         m.close()
         rows.append({"H": H, "us_p50": float(np.percentile(ms, 50)) * 1e3, "us_p10": float(np.percentile(ms, 10)) * 1e3,
                      "us_p90": float(np.percentile(ms, 90)) * 1e3, "rows_streamed": info["rows_streamed"],
-                     "threads": info["threads"], "max_rel_err": err})
+                     "threads": info["threads"], "batched_tensor_core": info.get("recur_batched_tensor_core"),
+                     "max_rel_err": err})
         print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
     hs = [r["H"] for r in rows]
     lat = [r["us_p50"] for r in rows]
-    res = {"workload": "cfg3 sweep: 1 layer, in = hidden = H, T = 35, B = 1, bf16 weights", "steps": args.steps, "points": rows}
+    label = ("ds2 sweep: 5 bidirectional layers, 1312 -> H, T = 400, B = 16, bf16 weights; us per call (16 utterances)" if ds2
+             else "cfg3 sweep: 1 layer, in = hidden = H, T = 35, B = 1, bf16 weights")
+    res = {"workload": label, "steps": args.steps, "points": rows}
     for eps in (0.0, 0.005):
         lhps, red = lhp_analysis(hs, lat, eps)
         res[f"lhp_eps_{eps:g}"] = {"lhps": lhps, "count": len(lhps), "redundancy_percent": red}
-    (outdir / "sweep_cfg3.json").write_text(json.dumps(res, indent=1))
+    (outdir / ("sweep_ds2_b16.json" if ds2 else "sweep_cfg3.json")).write_text(json.dumps(res, indent=1))
     print(json.dumps({k: v for k, v in res.items() if k != "points"}))
 
 
@@ -498,6 +519,7 @@ def main():
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--matmul-sweep", action="store_true")
     ap.add_argument("--sweep-sizes", default="")
+    ap.add_argument("--sweep-shape", default="cfg3", choices=["cfg3", "ds2"])
     ap.add_argument("--sweep-parity", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -84,6 +84,12 @@ def config5(B: int = 1) -> Workload:
     return Workload(f"cfg5_ds2_B{B}", 5, True, 1312, 800, 400, B, "bf16", 0.035, seed=_seed(5))
 
 
+def config5_width(H: int, B: int = 16) -> Workload:
+    """The speech-model shape at another hidden width (the width sweep of the paper's Figure 3): 5
+    bidirectional layers, 1312 -> H, then 2H -> H, T=400."""
+    return Workload(f"ds2_sweep_H{H}_B{B}", 5, True, 1312, H, 400, B, "bf16", 1.0 / math.sqrt(H), seed=_seed(5, H))
+
+
 def round_to_bf16(a: np.ndarray) -> np.ndarray:
     """float32 -> nearest-even bfloat16 -> float32 (finite inputs)."""
     a = np.ascontiguousarray(a, dtype=np.float32)

@@ -52,6 +52,7 @@ struct lstm_handle {
     bool use_mma = false;
     int mma_mt = 0, mma_nkr = 0, mma_nks = 0, mma_nw = 0;
     // batched tensor-core recurrence (more than four batch rows): weight-tile rows, K blocks, planes, stamps
+    bool seq_dirs = false;             // bidirectional layers run one direction after the other, each on all SMs
     bool use_tcb = false;
     int tcb_RA = 0, tcb_nkb = 0, tcb_ld = 0, tcb_ldh = 0, tcb_mapN = 0;
     __nv_bfloat16 *hplanes = nullptr; unsigned *tcb_flags = nullptr;
@@ -406,16 +407,30 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
     plan_mma(h);
-    {   // batched tensor-core recurrence: available beside the register-resident kernel when the slice fits
+    // does the batched tensor-core recurrence fit with the current split of the SMs?
+    auto tcb_fits = [&](int *kbs, int *stages) -> bool {
         const char *env = getenv("LSTM_B200_RECUR");
         const int RA = round_up(4 * h->upc, 8), nkb = (H + 63) / 64;
-        if (h->use_mma && max_B > 4 && RA <= 128 && !(env && strcmp(env, "mma") == 0)) {
-            const int B = std::min(max_B, 32), N = round_up(2 * B, 16);
-            int kbs = 0, stages = 0;
-            if (h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - 256, &kbs, &stages)) {
-                h->use_tcb = true; h->tcb_RA = RA; h->tcb_nkb = nkb; h->tcb_ld = nkb * 64; h->tcb_ldh = round_up(H, 8);
-            }
-        }
+        if (!(bf16 && !csr && max_B > 4 && RA <= 128) || (env && (strcmp(env, "mma") == 0 || strcmp(env, "simt") == 0))) return false;
+        const int B = std::min(max_B, 32), N = round_up(2 * B, 16);
+        return h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - 256, kbs, stages);
+    };
+    int kbs_tmp = 0, stages_tmp = 0;
+    if (D == 2 && bf16 && !csr && !h->use_mma && !tcb_fits(&kbs_tmp, &stages_tmp)) {
+        // Side by side, each direction has half the SMs and a slice twice as tall; when that slice fits
+        // neither the register-resident kernel nor (for handles made for batches) the tensor-core one, run
+        // the directions one after the other on all SMs instead: twice the steps, but every step on-chip.
+        const int nc = h->ncta_dir, up = h->upc, th = h->threads;
+        h->ncta_dir = std::max(1, std::min(h->sm_count, H));
+        h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
+        h->threads = std::max(128, 32 * std::min(h->upc, 16));
+        plan_mma(h);
+        if (h->use_mma) h->seq_dirs = true;
+        else { h->ncta_dir = nc; h->upc = up; h->threads = th; }
+    }
+    if (tcb_fits(&kbs_tmp, &stages_tmp)) {   // batched tensor-core recurrence, beside the kernels for up to four sequences
+        h->use_tcb = true; h->tcb_RA = round_up(4 * h->upc, 8); h->tcb_nkb = (H + 63) / 64; h->tcb_ld = h->tcb_nkb * 64;
+        h->tcb_ldh = round_up(H, 64);      // rows of the planes start on 128-byte lines: a TMA box row is one line, not two
     }
     h->layers.resize(layers);
     if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
@@ -492,20 +507,6 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                     }
                     rc = upload(h, (uint32_t **)&ly.wfrag[d], f.data(), f.size() * 4, st, "recurrent weight fragments");
                     if (rc == LSTM_OK) cudaStreamSynchronize(st);
-                    if (rc == LSTM_OK && h->use_tcb) {
-                        // the same slices as plain K-major rows for the tensor-core kernel's TMA tiles
-                        const size_t rows_dir = (size_t)h->ncta_dir * h->tcb_RA;
-                        if (d == 0) tcb_rows.assign((size_t)D * rows_dir * h->tcb_ld, 0);
-                        for (int c = 0; c < h->ncta_dir; ++c) {
-                            int u0, nu; unit_range_host(H, h->ncta_dir, c, u0, nu);
-                            for (int u = 0; u < nu; ++u)
-                                for (int q = 0; q < 4; ++q) {
-                                    const float *srow = m.data() + (size_t)(q * H + u0 + u) * H;
-                                    uint16_t *drow = tcb_rows.data() + ((size_t)d * rows_dir + (size_t)c * h->tcb_RA + 4 * u + q) * h->tcb_ld;
-                                    for (int k = 0; k < H; ++k) drow[k] = f32_to_bf16_rne(srow[k]);
-                                }
-                        }
-                    }
                 } else if (bf16) {
                     std::vector<uint16_t> p(n, 0);
                     for (int j = 0; j < H; ++j)
@@ -523,6 +524,20 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                             memcpy(p.data() + ((size_t)j * 4 + q) * h->Hp8, m.data() + (size_t)(q * H + j) * H, sizeof(float) * H);
                     rc = upload(h, &ly.wh[d], p.data(), n * 4, st, "recurrent weights");
                     if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                }
+                if (rc == LSTM_OK && h->use_tcb) {
+                    // the same slices as plain K-major rows for the tensor-core kernel's TMA tiles
+                    const size_t rows_dir = (size_t)h->ncta_dir * h->tcb_RA;
+                    if (d == 0) tcb_rows.assign((size_t)D * rows_dir * h->tcb_ld, 0);
+                    for (int c = 0; c < h->ncta_dir; ++c) {
+                        int u0, nu; unit_range_host(H, h->ncta_dir, c, u0, nu);
+                        for (int u = 0; u < nu; ++u)
+                            for (int q = 0; q < 4; ++q) {
+                                const float *srow = m.data() + (size_t)(q * H + u0 + u) * H;
+                                uint16_t *drow = tcb_rows.data() + ((size_t)d * rows_dir + (size_t)c * h->tcb_RA + 4 * u + q) * h->tcb_ld;
+                                for (int k = 0; k < H; ++k) drow[k] = f32_to_bf16_rne(srow[k]);
+                            }
+                    }
                 }
             } else {
                 HostCsr cx, ch;
@@ -885,7 +900,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
     cudaError_t e = cudaSuccess;
 
     // stamps of the exchange words must stay unique: restart from a cleared buffer before wrapping
-    if ((unsigned long long)h->stamp_next + (unsigned long long)L * T + 2ull >= 0xffffffffull) {
+    if ((unsigned long long)h->stamp_next + (unsigned long long)L * D * ((unsigned long long)T + 1ull) + 2ull >= 0xffffffffull) {
         if (cudaMemsetAsync(h->xch, 0, h->xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->rxch && cudaMemsetAsync(h->rxch, 0, h->rxch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->tcb_flags && cudaMemsetAsync(h->tcb_flags, 0, (size_t)D * h->ncta_dir * sizeof(unsigned), st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
@@ -900,10 +915,13 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         // ---- input staging + projection
         { const int prc = run_projection(h, l, l == 0 ? x : nullptr, Xf, M, N, &nsplit, st); if (prc != LSTM_OK) return prc; }
 
-        // ---- recurrence
+        // ---- recurrence: all directions in one launch, or one launch per direction
+        const int npass = h->seq_dirs ? D : 1;
+        for (int pass = 0; pass < npass; ++pass) {
         if (h->Hh) {
             HlstmArgs m;
             memset(&m, 0, sizeof m);
+            m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
             m.H = H; m.Hh = h->Hh; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
             m.nks1 = h->mma_nks; m.nkw2 = h->hl_nkw2;
             m.stamp_base = h->stamp_next;
@@ -934,6 +952,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (h->use_tcb && B > 4 && B <= 32) {
             RecurTcArgs m;
             memset(&m, 0, sizeof m);
+            m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
             m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
             m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16);
             if (!recur_tc_plan(m.RA, m.nkb, m.N, h->upc, B, (size_t)h->smem_optin - 256, &m.kbs, &m.stages))
@@ -972,6 +991,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (h->use_mma) {
             RecurMmaArgs m;
             memset(&m, 0, sizeof m);
+            m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
             m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit; m.nkw_smem = h->mma_nks; m.staged = shp.staged ? 1 : 0;
             m.stamp_base = h->stamp_next;
             h->stamp_next += (unsigned)T + 1u;
@@ -998,6 +1018,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         }
         RecurArgs a;
         memset(&a, 0, sizeof a);
+        a.dir0 = h->seq_dirs ? pass : 0; a.ndirs = h->seq_dirs ? 1 : D;
         a.H = H; a.Hp8 = h->Hp8; a.Hs = h->Hs; a.B = B; a.T = T; a.D = D;
         a.ncta_dir = h->ncta_dir; a.nsplit = nsplit; a.BT = shp.BT; a.w_smem_bytes = shp.w_smem_bytes;
         a.stamp_base = h->stamp_next;
@@ -1021,6 +1042,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         ++h->last_launches;
         if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
         if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
+        }
     }
     return LSTM_OK;
 }

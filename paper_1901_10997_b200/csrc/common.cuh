@@ -16,6 +16,7 @@ constexpr int kStatusTimeout = 5;
 // evenly over a direction's CTAs; CTA c owns units [u0(c), u0(c) + n(c)).
 // ---------------------------------------------------------------------------------------------------
 struct RecurArgs {
+    int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
     int H;              // hidden width
     int Hp8;            // dense: row length of the packed recurrent matrix (H rounded up to 8)
     int Hs;             // length of one staged h row in shared memory (H rounded up to 256)
@@ -59,6 +60,7 @@ cudaError_t recur_csr_prepare(int max_smem);
 // tile, the first NKR of them in registers, the remaining nkw_smem in shared memory.
 // ---------------------------------------------------------------------------------------------------
 struct RecurMmaArgs {
+    int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
     int H, B, T, D;
     int ncta_dir;
     int nsplit;
@@ -95,6 +97,7 @@ cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, siz
 // 2b+1 = lo part of batch row b) and one stamp per producer CTA.
 // ---------------------------------------------------------------------------------------------------
 struct RecurTcArgs {
+    int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
     int H, B, T, D;
     int ncta_dir;
     int nsplit;
@@ -133,6 +136,7 @@ cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurT
 // CTAs, fragments in shared memory).  Fragment layout as in RecurMmaArgs.
 // ---------------------------------------------------------------------------------------------------
 struct HlstmArgs {
+    int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
     int H, Hh, B, T, D;
     int ncta_dir;
     int nsplit;

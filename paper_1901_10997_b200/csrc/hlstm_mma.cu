@@ -133,8 +133,8 @@ __global__ void __launch_bounds__(NW * 32, 1) hlstm_mma_kernel(const HlstmArgs a
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tig = lane & 3;
     const int H = a.H, Hh = a.Hh, B = a.B, T = a.T, D = a.D;
-    const int d = blockIdx.x / a.ncta_dir;
-    const int cta = blockIdx.x - d * a.ncta_dir;
+    const int d = a.dir0 + blockIdx.x / a.ncta_dir;
+    const int cta = blockIdx.x % a.ncta_dir;
     int m0, nm, u0, nu;
     unit_range(Hh, a.ncta_dir, cta, m0, nm);       // hidden units of this CTA (pass 1)
     unit_range(H, a.ncta_dir, cta, u0, nu);        // cell units of this CTA (pass 2)
@@ -391,7 +391,7 @@ cudaError_t launch_hlstm_mma(const HlstmArgs &a, int mt, int nkr, int nw, size_t
     if (!fn) return cudaErrorInvalidValue;
     HlstmArgs copy = a;
     void *params[] = {&copy};
-    return cudaLaunchCooperativeKernel((const void *)fn, dim3(a.ncta_dir * a.D), dim3(nw * 32), params, smem, st);
+    return cudaLaunchCooperativeKernel((const void *)fn, dim3(a.ncta_dir * (a.ndirs ? a.ndirs : a.D)), dim3(nw * 32), params, smem, st);
 }
 
 }  // namespace lstm

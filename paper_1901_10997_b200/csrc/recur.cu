@@ -205,8 +205,8 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nthreads = blockDim.x, nwarps = nthreads >> 5;
     const int H = a.H, Hs = a.Hs, B = a.B, T = a.T, D = a.D;
-    const int d = blockIdx.x / a.ncta_dir;
-    const int cta = blockIdx.x - d * a.ncta_dir;
+    const int d = a.dir0 + blockIdx.x / a.ncta_dir;
+    const int cta = blockIdx.x % a.ncta_dir;
     int u0, nu;
     unit_range(H, a.ncta_dir, cta, u0, nu);
     const int upc = (H + a.ncta_dir - 1) / a.ncta_dir;
@@ -416,7 +416,7 @@ cudaError_t launch_bt(const RecurArgs &a, int threads, size_t smem, cudaStream_t
     }
     RecurArgs copy = a;
     void *params[] = {&copy};
-    return cudaLaunchCooperativeKernel(fn, dim3(a.ncta_dir * a.D), dim3(threads), params, smem, st);
+    return cudaLaunchCooperativeKernel(fn, dim3(a.ncta_dir * (a.ndirs ? a.ndirs : a.D)), dim3(threads), params, smem, st);
 }
 
 template <bool BF16, bool CSR>

@@ -109,8 +109,8 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tig = lane & 3;
     const int H = a.H, B = a.B, T = a.T, D = a.D;
-    const int d = blockIdx.x / a.ncta_dir;
-    const int cta = blockIdx.x - d * a.ncta_dir;
+    const int d = a.dir0 + blockIdx.x / a.ncta_dir;
+    const int cta = blockIdx.x % a.ncta_dir;
     int u0, nu;
     unit_range(H, a.ncta_dir, cta, u0, nu);
     const int upc = (H + a.ncta_dir - 1) / a.ncta_dir;
@@ -451,7 +451,7 @@ cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, siz
     if (!fn) return cudaErrorInvalidValue;
     RecurMmaArgs copy = a;
     void *params[] = {&copy};
-    return cudaLaunchCooperativeKernel((const void *)fn, dim3(a.ncta_dir * a.D), dim3(nw * 32), params, smem, st);
+    return cudaLaunchCooperativeKernel((const void *)fn, dim3(a.ncta_dir * (a.ndirs ? a.ndirs : a.D)), dim3(nw * 32), params, smem, st);
 }
 
 }  // namespace lstm

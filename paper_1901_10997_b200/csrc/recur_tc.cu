@@ -164,8 +164,8 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int H = a.H, B = a.B, T = a.T, D = a.D, N = a.N, S = a.stages, RA = a.RA, nkb = a.nkb, kbs = a.kbs;
-    const int d = blockIdx.x / a.ncta_dir;
-    const int cta = blockIdx.x - d * a.ncta_dir;
+    const int d = a.dir0 + blockIdx.x / a.ncta_dir;
+    const int cta = blockIdx.x % a.ncta_dir;
     int u0, nu;
     unit_range(H, a.ncta_dir, cta, u0, nu);
     const int upc = (H + a.ncta_dir - 1) / a.ncta_dir;
@@ -505,7 +505,7 @@ cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurT
     memcpy(&mh, tmap_h, sizeof mh);
     RecurTcArgs copy = a;
     void *params[] = {&mw, &mh, &copy};
-    return cudaLaunchCooperativeKernel((const void *)recur_tc_kernel, dim3(a.ncta_dir * a.D), dim3(kThreads), params, smem, st);
+    return cudaLaunchCooperativeKernel((const void *)recur_tc_kernel, dim3(a.ncta_dir * (a.ndirs ? a.ndirs : a.D)), dim3(kThreads), params, smem, st);
 }
 
 }  // namespace lstm

@@ -241,6 +241,25 @@ def test_batched_tensor_core_recurrence(oracle, w):
     m.close()
 
 
+@pytest.mark.parametrize("B", [2, 9])
+def test_wide_bidirectional_stack_runs_its_directions_one_after_the_other(oracle, B):
+    """At this width half the SMs cannot hold one direction's slice on-chip, so the handle gives each
+    direction all SMs in turn (148 CTAs per direction instead of 74); results are the same stack."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = small("seq_dirs", 2, True, 40, 1500, 3, B, "bf16", scale=0.03, seed=31)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=2, bidir=True, hidden=w.hidden)
+    m = pkg.LSTM(weights, layers=2, in_dim=w.in_dim, hidden=w.hidden, bidir=True, dtype="bf16", max_T=w.T, max_B=B)
+    info = m.info()
+    assert info["ctas_per_dir"] == info["sm_count"] and info["recur_register_resident"] == 1
+    y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
+    m.check()
+    assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"seq dirs B={B}")
+    m.close()
+
+
 def test_batched_recurrence_chunked_calls_carry_state(oracle):
     w = small("tc_chunk", 2, True, 24, 150, 9, 8, "bf16", seed=9)
     weights, x = wl.make(w)
