@@ -239,16 +239,22 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             long long t_start = 0;
             int rounds = 0;
             bool aborted = false;
+            bool seen[kFlagLoads];
+#pragma unroll
+            for (int k = 0; k < kFlagLoads; ++k) seen[k] = lane + 32 * k >= a.ncta_dir;
             while (true) {
+                // only the stamps not yet seen are asked for again: most producers are early, and the lines
+                // that hold the stamps are the busiest in the L2 (every CTA reads and writes them)
                 unsigned v[kFlagLoads];
 #pragma unroll
-                for (int k = 0; k < kFlagLoads; ++k) {
-                    const int i = lane + 32 * k;
-                    v[k] = i < a.ncta_dir ? ld_relaxed_u32(flags_d + i) : want;
-                }
+                for (int k = 0; k < kFlagLoads; ++k)
+                    if (!seen[k]) v[k] = ld_relaxed_u32(flags_d + lane + 32 * k);
                 bool ok = true;
 #pragma unroll
-                for (int k = 0; k < kFlagLoads; ++k) ok &= (int)(v[k] - want) >= 0;
+                for (int k = 0; k < kFlagLoads; ++k) {
+                    if (!seen[k]) seen[k] = (int)(v[k] - want) >= 0;
+                    ok &= seen[k];
+                }
                 // both votes are taken by all lanes every round, so the warp leaves the loop as one
                 if (__any_sync(0xffffffffu, *abort_flag != 0)) { aborted = true; break; }
                 if (__all_sync(0xffffffffu, ok)) break;
