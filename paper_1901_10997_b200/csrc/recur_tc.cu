@@ -129,6 +129,8 @@ __device__ __forceinline__ float4 ld_nc_f4(const float4 *p)
     asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
     return v;
 }
+// release / acquire fence at GPU scope (lighter than the sequentially consistent __threadfence)
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ void st_relaxed_u32(unsigned *p, unsigned v)
 {
     asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -265,7 +267,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                 }
             }
             if (aborted) break;
-            __threadfence();                                        // acquire: the planes behind the stamps
+            fence_acq_rel_gpu();                                    // acquire: the planes behind the stamps
             asm volatile("fence.proxy.async;" ::: "memory");       // they were written with ordinary stores
             const int row0 = (d * 2 + ((s + 1) & 1)) * 64;          // planes of step s-1 live in parity (s-1)&1
             for (int g0 = 0; g0 < nkb; g0 += kbs) {
@@ -329,7 +331,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         bar_sync(1, 128);
         if (ftid == 0) {
             if ((int)blockIdx.x != a.withhold_cta) {
-                __threadfence();
+                fence_acq_rel_gpu();
                 st_relaxed_u32(flags_d + cta, a.stamp_base);
             }
             *pub = 1;
@@ -416,7 +418,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             bar_sync(1, 128);
             if (ftid == 0) {
                 if ((int)blockIdx.x != a.withhold_cta) {
-                    __threadfence();
+                    fence_acq_rel_gpu();
                     st_relaxed_u32(flags_d + cta, a.stamp_base + (unsigned)s + 1u);
                 }
                 *pub = s + 2;
