@@ -54,6 +54,7 @@ struct lstm_handle {
     // batched tensor-core recurrence (more than four batch rows): weight-tile rows, K blocks, planes, stamps
     bool seq_dirs = false;             // bidirectional layers run one direction after the other, each on all SMs
     bool use_tcb = false;
+    bool tcb_pair = false;             // the batched recurrence splits K over clusters of two CTAs
     int tcb_RA = 0, tcb_nkb = 0, tcb_ld = 0, tcb_ldh = 0, tcb_mapN = 0;
     __nv_bfloat16 *hplanes = nullptr; unsigned *tcb_flags = nullptr;
     alignas(64) unsigned char tmap_planes[128];
@@ -413,7 +414,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
         const int RA = round_up(4 * h->upc, 8), nkb = (H + 63) / 64;
         if (!(bf16 && !csr && max_B > 4 && RA <= 128) || (env && (strcmp(env, "mma") == 0 || strcmp(env, "simt") == 0))) return false;
         const int B = std::min(max_B, 32), N = round_up(2 * B, 16);
-        return h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - 256, kbs, stages);
+        return h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - 256, 0, kbs, stages);
     };
     int kbs_tmp = 0, stages_tmp = 0;
     if (D == 2 && bf16 && !csr && !h->use_mma && !tcb_fits(&kbs_tmp, &stages_tmp)) {
@@ -431,6 +432,16 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     if (tcb_fits(&kbs_tmp, &stages_tmp)) {   // batched tensor-core recurrence, beside the kernels for up to four sequences
         h->use_tcb = true; h->tcb_RA = round_up(4 * h->upc, 8); h->tcb_nkb = (H + 63) / 64; h->tcb_ld = h->tcb_nkb * 64;
         h->tcb_ldh = round_up(H, 64);      // rows of the planes start on 128-byte lines: a TMA box row is one line, not two
+        // pair mode: two CTAs of a cluster split K (half the tensor instructions per step) when the pairs do
+        // not straddle directions, the doubled tile fits, and the device can co-schedule the clusters
+        const char *env = getenv("LSTM_B200_RECUR");
+        const int Bp = std::min(max_B, 32), Np = round_up(2 * Bp, 16);
+        int kp = 0, sp = 0;
+        if (!(env && strcmp(env, "tc1") == 0) && (h->ncta_dir % 2) == 0 &&
+            recur_tc_plan(h->tcb_RA, h->tcb_nkb, Np, h->upc, Bp, (size_t)h->smem_optin - 256, 1, &kp, &sp) &&
+            recur_tc_prepare(h->smem_optin - 256) == cudaSuccess &&
+            recur_tc_pair_supported(h->ncta_dir * (h->seq_dirs ? 1 : D), recur_tc_smem_bytes(h->tcb_RA, h->tcb_nkb, Np, sp, kp, h->upc, Bp, 1)))
+            h->tcb_pair = true;
     }
     h->layers.resize(layers);
     if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
@@ -586,7 +597,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
         rc = upload(h, &ly.bias, bias_p.data(), bias_p.size() * 4, st, "bias");
         if (rc == LSTM_OK && h->use_tcb && !tcb_rows.empty()) {
             rc = upload(h, (uint16_t **)&ly.wtc, tcb_rows.data(), tcb_rows.size() * 2, st, "recurrent weight tiles");
-            if (rc == LSTM_OK && !recur_tc_encode_weights(ly.tmap_wtc, ly.wtc, (long long)D * h->ncta_dir * h->tcb_RA, h->tcb_ld, h->tcb_RA))
+            if (rc == LSTM_OK && !recur_tc_encode_weights(ly.tmap_wtc, ly.wtc, (long long)D * h->ncta_dir * h->tcb_RA, h->tcb_ld, h->tcb_pair ? 2 * h->tcb_RA : h->tcb_RA))
                 rc = fail(h, LSTM_ERR_CUDA, "tensor map of the recurrent weight tiles could not be encoded");
         }
         if (rc == LSTM_OK && !csr)
@@ -955,7 +966,8 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
             m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
             m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16);
-            if (!recur_tc_plan(m.RA, m.nkb, m.N, h->upc, B, (size_t)h->smem_optin - 256, &m.kbs, &m.stages))
+            m.pair = h->tcb_pair ? 1 : 0;
+            if (!recur_tc_plan(m.RA, m.nkb, m.N, h->upc, B, (size_t)h->smem_optin - 256, m.pair, &m.kbs, &m.stages))
                 return fail(h, LSTM_ERR_INVALID, "batched recurrence does not fit shared memory at batch %d", B);
             m.tmem_cols = m.N <= 32 ? 32 : 64;
             m.ldh = h->tcb_ldh;
@@ -979,7 +991,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
                     return fail(h, LSTM_ERR_CUDA, "tensor map of the h planes could not be encoded");
                 h->tcb_mapN = m.N;
             }
-            const size_t smem = recur_tc_smem_bytes(m.RA, m.nkb, m.N, m.stages, m.kbs, h->upc, B);
+            const size_t smem = recur_tc_smem_bytes(m.RA, m.nkb, m.N, m.stages, m.kbs, h->upc, B, m.pair);
             if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
             e = launch_recur_tc(ly.tmap_wtc, h->tmap_planes, m, smem, st);
             ++h->last_launches;

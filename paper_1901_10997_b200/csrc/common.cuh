@@ -105,6 +105,7 @@ struct RecurTcArgs {
     int N;                      // MMA N: 2 * B rounded up to 16
     int stages;                 // depth of the operand ring
     int kbs;                    // K blocks per ring stage
+    int pair;                   // 1: clusters of two CTAs split K (launched with cluster dimension 2)
     int tmem_cols;              // power of two >= max(32, N)
     int ldh;                    // row stride of the planes (elements, multiple of 8)
     unsigned stamp_base;
@@ -122,8 +123,9 @@ struct RecurTcArgs {
     unsigned *flags;            // [D][ncta_dir]
     int *status;
 };
-size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc, int B);
-bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int *kbs_out, int *stages_out);
+size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc, int B, int pair);
+bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int pair, int *kbs_out, int *stages_out);
+bool recur_tc_pair_supported(int grid, size_t smem);
 bool recur_tc_encode_weights(void *map128, const void *w, long long rows, int ld, int RA);
 bool recur_tc_encode_planes(void *map128, const void *hbuf, int D, int H, int ldh, int N);
 cudaError_t recur_tc_prepare(int max_smem);

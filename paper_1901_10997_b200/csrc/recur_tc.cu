@@ -21,6 +21,13 @@
 //   warps 2-5 request their projection terms, then read the accumulator rows of the CTA's units back
 //            (tcgen05.ld), add hi and lo columns, and finish the (unit, batch row) pairs: gates, c/h update,
 //            outputs, and the new h as bf16 planes; then one thread fences and raises the CTA's stamp.
+// Pair mode (chosen at create time when the CTA count per direction is even, the doubled tile fits and the
+// device can co-schedule the clusters): CTAs 2p and 2p+1 are launched as a cluster of two; each keeps the
+// weight rows of BOTH CTAs' units but only half of the K blocks, so each issues half the tensor
+// instructions per step; the partial sums of the partner's units go to the partner's shared memory
+// (st.shared::cluster) followed by a release arrive on the partner's mbarrier, and every CTA finishes its
+// own units from its own and the received partial sums.  The wait for the partner is bounded like the rest,
+// and a cluster barrier at the common exit keeps a CTA resident while its partner may still write into it.
 // Every wait (stamps, mbarriers) is bounded; on expiry the CTA records a timeout status and all roles fall
 // through to the common exit where tensor memory is released.  No TMA multicast is used.
 #include "common.cuh"
@@ -141,6 +148,58 @@ __device__ __forceinline__ int ld_volatile_s32(const int *p)
     asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// ---- two-CTA cluster helpers (pair mode): the partner's shared memory and barriers
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t remote_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_acquire_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait for the partner's arrival; false when it gave up or another role did.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    long long t_start = 0;
+    for (long long it = 0;; ++it) {
+        if (mbar_try_wait_acquire_cluster(bar, parity)) return true;
+        if ((it & 255) == 255) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t_start == 0) t_start = now;
+            if (now - t_start > kWaitTicks) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
 __device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
@@ -160,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h, const RecurTcArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar, w_bar;
+    __shared__ __align__(8) unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar, w_bar, partial_bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s, pub_s;
 
@@ -171,15 +230,26 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     int u0, nu;
     unit_range(H, a.ncta_dir, cta, u0, nu);
     const int upc = (H + a.ncta_dir - 1) / a.ncta_dir;
+    // Pair mode: CTAs 2p and 2p+1 form a cluster; each keeps the rows of BOTH CTAs' units (RT = 2 RA rows) but
+    // only half of the K blocks, multiplies its half, and hands the partner the partial sums of the partner's
+    // units through distributed shared memory: half the tensor instructions per step and CTA.
+    const int pair = a.pair;
+    const int rank = pair ? (int)cluster_ctarank() : 0;
+    const int RT = pair ? 2 * RA : RA;                                      // rows of a weight tile
+    const int nkb_half = (nkb + 1) / 2;
+    const int kb_lo = (pair && rank) ? nkb_half : 0;                        // first K block of this CTA
+    const int nkb_my = pair ? (rank ? nkb - nkb_half : nkb_half) : nkb;     // K blocks of this CTA
+    const int nkb_alloc = pair ? nkb_half : nkb;                            // same layout in both CTAs of a pair
 
     // shared-memory carve-up (tiles need 1024-byte alignment): weight tiles, operand ring, then scratch
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_tiles = base;                                          // [nkb][RA rows][128 B]
-    const uint32_t ring = a_tiles + (uint32_t)nkb * RA * 128;               // [S][kbs][N rows][128 B]
+    const uint32_t a_tiles = base;                                          // [nkb_alloc][RT rows][128 B]
+    const uint32_t ring = a_tiles + (uint32_t)nkb_alloc * RT * 128;         // [S][kbs][N rows][128 B]
     unsigned char *gen = smem_raw + (ring + (uint32_t)(S * kbs * N) * 128 - smem_u32(smem_raw));
     float *zs = reinterpret_cast<float *>(gen);                             // [B][4*upc] gate pre-activations (h part)
     const int zld = 4 * upc;
     float *c_s = zs + zld * B;                                              // [B][units of this CTA]
+    float *zs2 = c_s + ((upc * B + 3) & ~3);                                // [B][4*upc] the partner's partial sums (pair mode)
 
     if (tid == 0) {
         abort_s = 0;
@@ -187,6 +257,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
         mbar_init(smem_u32(&accum_bar), 1);
         mbar_init(smem_u32(&w_bar), 1);
+        mbar_init(smem_u32(&partial_bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -202,6 +273,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (pair) cluster_sync_all();               // the partner's barriers are initialised before anything reaches them
     const uint32_t tmem_base = tmem_base_s;
     volatile int *abort_flag = &abort_s;
     volatile int *pub = &pub_s;                 // steps this CTA has published (h0 counts as one)
@@ -212,10 +284,11 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     if (warp == 0) {
         // ================= stamps and TMA =================
         // the CTA's weight tiles, once (one lane per tile)
-        if (lane == 0) mbar_expect_tx(smem_u32(&w_bar), (uint32_t)nkb * RA * 128);
+        if (lane == 0) mbar_expect_tx(smem_u32(&w_bar), (uint32_t)nkb_my * RT * 128);
         __syncwarp();
-        for (int kb = lane; kb < nkb; kb += 32)
-            tma_load_2d(a_tiles + (uint32_t)kb * RA * 128, &tmap_w, smem_u32(&w_bar), kb * 64, (d * a.ncta_dir + cta) * RA);
+        for (int kb = lane; kb < nkb_my; kb += 32)
+            tma_load_2d(a_tiles + (uint32_t)kb * RT * 128, &tmap_w, smem_u32(&w_bar), (kb_lo + kb) * 64,
+                        (d * a.ncta_dir + (pair ? (cta & ~1) : cta)) * RA);
         // ring position as a stage index and a phase bit (a 64-bit divide per stage would cost the issuing
         // thread more than the copies it issues)
         int st = 0;
@@ -270,8 +343,8 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             fence_acq_rel_gpu();                                    // acquire: the planes behind the stamps
             asm volatile("fence.proxy.async;" ::: "memory");       // they were written with ordinary stores
             const int row0 = (d * 2 + ((s + 1) & 1)) * 64;          // planes of step s-1 live in parity (s-1)&1
-            for (int g0 = 0; g0 < nkb; g0 += kbs) {
-                const int nblk = min(kbs, nkb - g0);
+            for (int g0 = 0; g0 < nkb_my; g0 += kbs) {
+                const int nblk = min(kbs, nkb_my - g0);
                 int ok = 1;
                 if (lane == 0) {
                     ok = mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abort_flag) ? 1 : 0;
@@ -281,7 +354,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                 if (!ok) { live = false; break; }
                 // one lane per K block of the stage: issuing a tensor copy occupies a thread for a while
                 if (lane < nblk)
-                    tma_load_2d(ring + (uint32_t)((st * kbs + lane) * N) * 128, &tmap_h, smem_u32(&full_bar[st]), (g0 + lane) * 64, row0);
+                    tma_load_2d(ring + (uint32_t)((st * kbs + lane) * N) * 128, &tmap_h, smem_u32(&full_bar[st]), (kb_lo + g0 + lane) * 64, row0);
                 if (++st == S) { st = 0; ph ^= 1u; }
             }
         }
@@ -292,13 +365,13 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             bool ok = mbar_wait(smem_u32(&w_bar), 0u, abort_flag);
             // descriptors differ only in their start-address field (units of 16 bytes): build one of each and add
             const uint64_t adesc0 = umma_desc_sw128(a_tiles), bdesc0 = umma_desc_sw128(ring);
-            const uint32_t a_step = (uint32_t)(RA * 128) >> 4, b_step = (uint32_t)(N * 128) >> 4;
+            const uint32_t a_step = (uint32_t)(RT * 128) >> 4, b_step = (uint32_t)(N * 128) >> 4;
             int st = 0;
             uint32_t ph = 0;
             for (int s = 0; s < T && ok; ++s) {
                 uint64_t adesc = adesc0;
-                for (int g0 = 0; g0 < nkb; g0 += kbs) {
-                    const int nblk = min(kbs, nkb - g0);
+                for (int g0 = 0; g0 < nkb_my; g0 += kbs) {
+                    const int nblk = min(kbs, nkb_my - g0);
                     ok = mbar_wait(smem_u32(&full_bar[st]), ph, abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -319,6 +392,13 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         const int ftid = tid - 64;                       // 0..127
         const int lq = warp & 3;                         // TMEM lane quadrant this warp may read
         const int nuB = nu * B;
+        int u0_partner = 0, nu_partner = 0;
+        uint32_t zs2_remote = 0, partial_bar_remote = 0;
+        if (pair) {
+            unit_range(H, a.ncta_dir, cta ^ 1, u0_partner, nu_partner);
+            zs2_remote = map_to_cta(smem_u32(zs2), (uint32_t)(rank ^ 1));
+            partial_bar_remote = map_to_cta(smem_u32(&partial_bar), (uint32_t)(rank ^ 1));
+        }
         // the planes of h0 (stamp_base): this CTA's units
         for (int p = ftid; p < nuB; p += 128) {
             const int b = p / nu, u = p - b * nu;
@@ -354,23 +434,38 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             }
             if (!mbar_wait(smem_u32(&accum_bar), (uint32_t)s & 1u, abort_flag)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int row = lq * 32 + lane;              // accumulator row = 4 * unit + gate
-            if (lq * 32 < 4 * nu) {
+            // accumulator row = 4 * unit + gate; in pair mode rows [0, RA) belong to the even CTA's units and
+            // rows [RA, 2 RA) to the odd CTA's: the partner's rows go to the partner's shared memory
+            const int row = lq * 32 + lane;
+            const int half = (pair && row >= RA) ? 1 : 0;
+            const int lr = row - half * RA;
+            const bool mine = !pair || half == rank;
+            const bool row_ok = row < RT && lr < 4 * (mine ? nu : nu_partner);
+            if (lq * 32 < (pair ? RT : 4 * nu)) {
                 for (int c0 = 0; c0 < 2 * B; c0 += 16) {
                     uint32_t v[16];
                     tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (row < 4 * nu) {
+                    if (row_ok) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const int b = (c0 >> 1) + i;
-                            if (b < B) zs[b * zld + row] = __uint_as_float(v[2 * i]) + __uint_as_float(v[2 * i + 1]);
+                            const float z = __uint_as_float(v[2 * i]) + __uint_as_float(v[2 * i + 1]);
+                            if (b < B) {
+                                if (mine) zs[b * zld + lr] = z;
+                                else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                            }
                         }
                     }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             bar_sync(1, 128);
+            if (pair) {
+                // tell the partner its partial sums are in place, then wait for ours (bounded)
+                if (ftid == 0) mbar_arrive_remote_release(partial_bar_remote);
+                if (!mbar_wait_cluster(smem_u32(&partial_bar), (uint32_t)s & 1u, abort_flag)) break;
+            }
             __nv_bfloat16 *hp = hbuf_d + (size_t)(s & 1) * 64 * a.ldh;
             for (int i = 0; ftid + 128 * i < nuB; ++i) {
                 const int p = ftid + 128 * i;
@@ -392,7 +487,11 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                         gsum.x += g4.x; gsum.y += g4.y; gsum.z += g4.z; gsum.w += g4.w;
                     }
                 }
-                const float4 z4 = *reinterpret_cast<const float4 *>(zs + b * zld + 4 * u);
+                float4 z4 = *reinterpret_cast<const float4 *>(zs + b * zld + 4 * u);
+                if (pair) {
+                    const float4 y4 = *reinterpret_cast<const float4 *>(zs2 + b * zld + 4 * u);
+                    z4.x += y4.x; z4.y += y4.y; z4.z += y4.z; z4.w += y4.w;
+                }
                 const float gi = sigmoid_fast(z4.x + gsum.x);
                 const float gf = sigmoid_fast(z4.y + gsum.y);
                 const float gg = tanh_fast(z4.z + gsum.z);
@@ -432,6 +531,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
     }
     if (tid == 0 && abort_s) atomicExch(a.status, kStatusTimeout);
+    if (pair) cluster_sync_all();               // no CTA leaves while its partner may still write into its shared memory
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -467,22 +567,27 @@ bool encode_2d(void *map, const void *base, long long rows, int cols, int ld, in
 
 static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
 
-size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc, int B)
+size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc, int B, int pair)
 {
-    // the last weight tile is read as 128 rows: at least (128 - RA) * 128 bytes must follow it
-    const size_t after = (size_t)stages * kbs * N * 128 + (size_t)(4 * upc * B + upc * B) * 4 + 16;
-    const size_t need = (size_t)(128 - RA) * 128;
-    return 1024 + (size_t)nkb * RA * 128 + (after > need ? after : need);
+    // pair mode: tiles of 2 RA rows, half of the K blocks (rounded up), and a second block of partial sums
+    const int RT = pair ? 2 * RA : RA, nkb_alloc = pair ? (nkb + 1) / 2 : nkb;
+    // the last weight tile is read as 128 rows: at least (128 - RT) * 128 bytes must follow it
+    const size_t scratch = (size_t)(4 * upc * B) * (pair ? 2 : 1) + (size_t)((upc * B + 3) & ~3);
+    const size_t after = (size_t)stages * kbs * N * 128 + scratch * 4 + 16;
+    const size_t need = (size_t)(128 - RT) * 128;
+    return 1024 + (size_t)nkb_alloc * RT * 128 + (after > need ? after : need);
 }
 
 // Ring shape for one launch: stages of up to four K blocks (one mbarrier round trip per stage instead of per
 // block), as many stages as fit, at least two unless one stage holds the whole operand.
-bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int *kbs_out, int *stages_out)
+bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int pair, int *kbs_out, int *stages_out)
 {
-    for (int kbs = nkb < 4 ? nkb : 4; kbs >= 1; --kbs) {
-        const int groups = (nkb + kbs - 1) / kbs;
+    const int nkb_cta = pair ? (nkb + 1) / 2 : nkb;
+    if (pair && (2 * RA > 128 || nkb < 2)) return false;
+    for (int kbs = nkb_cta < 4 ? nkb_cta : 4; kbs >= 1; --kbs) {
+        const int groups = (nkb_cta + kbs - 1) / kbs;
         for (int st = groups < kMaxStages ? groups : kMaxStages; st >= (groups > 1 ? 2 : 1); --st) {
-            if (recur_tc_smem_bytes(RA, nkb, N, st, kbs, upc, B) <= max_smem) {
+            if (recur_tc_smem_bytes(RA, nkb, N, st, kbs, upc, B, pair) <= max_smem) {
                 *kbs_out = kbs;
                 *stages_out = st;
                 return true;
@@ -506,6 +611,25 @@ cudaError_t recur_tc_prepare(int max_smem)
     return cudaFuncSetAttribute(recur_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
 }
 
+// Can `grid` CTAs of this kernel be co-resident as clusters of two (pair mode needs every pair on one GPC)?
+bool recur_tc_pair_supported(int grid, size_t smem)
+{
+    if (grid < 2 || (grid & 1)) return false;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, (const void *)recur_tc_kernel, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return clusters * 2 >= grid;
+}
+
 cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurTcArgs &a, size_t smem, cudaStream_t st)
 {
     CUtensorMap mw, mh;
@@ -513,7 +637,19 @@ cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurT
     memcpy(&mh, tmap_h, sizeof mh);
     RecurTcArgs copy = a;
     void *params[] = {&mw, &mh, &copy};
-    return cudaLaunchCooperativeKernel((const void *)recur_tc_kernel, dim3(a.ncta_dir * (a.ndirs ? a.ndirs : a.D)), dim3(kThreads), params, smem, st);
+    const int grid = a.ncta_dir * (a.ndirs ? a.ndirs : a.D);
+    if (!a.pair)
+        return cudaLaunchCooperativeKernel((const void *)recur_tc_kernel, dim3(grid), dim3(kThreads), params, smem, st);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    return cudaLaunchKernelExC(&cfg, (const void *)recur_tc_kernel, params);
 }
 
 }  // namespace lstm
