@@ -165,7 +165,7 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def oracle_time(w: wl.Workload, weights, x, target_seconds=12.0, max_reps=50, mode="dense"):
+def oracle_time(w: wl.Workload, weights, x, target_seconds=12.0, max_reps=400, mode="dense"):
     """Times the oracle as it stands on a bounded sample: whole sequences of the workload (for B > 1
     only the first batch column), repeated until ~target_seconds of wall time have passed."""
     import oracle
