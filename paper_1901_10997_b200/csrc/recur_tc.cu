@@ -442,18 +442,25 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             const bool mine = !pair || half == rank;
             const bool row_ok = row < RT && lr < 4 * (mine ? nu : nu_partner);
             if (lq * 32 < (pair ? RT : 4 * nu)) {
-                for (int c0 = 0; c0 < 2 * B; c0 += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0, v);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (row_ok) {
+                // all column chunks are requested before the one wait (N <= 64: at most four chunks of 16)
+                uint32_t v[4][16];
+                const int nchunk = (2 * B + 15) >> 4;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int b = (c0 >> 1) + i;
-                            const float z = __uint_as_float(v[2 * i]) + __uint_as_float(v[2 * i + 1]);
-                            if (b < B) {
-                                if (mine) zs[b * zld + lr] = z;
-                                else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                for (int c = 0; c < 4; ++c)
+                    if (c < nchunk) tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(c * 16), v[c]);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row_ok) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < nchunk) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const int b = c * 8 + i;
+                                const float z = __uint_as_float(v[c][2 * i]) + __uint_as_float(v[c][2 * i + 1]);
+                                if (b < B) {
+                                    if (mine) zs[b * zld + lr] = z;
+                                    else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                                }
                             }
                         }
                     }
