@@ -344,3 +344,27 @@ def test_random_shapes(oracle, c):
     ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
     got = run_gpu(w, weights, x, h0, c0, exec_mode=c["mode"])
     assert_close(got, ref, w.dtype, "fuzz")
+
+
+def _fuzz_batched(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        H = int(rng.choice([rng.integers(8, 150), rng.integers(150, 700), rng.integers(700, 1700)]))
+        cases.append(dict(L=int(rng.integers(1, 3)), bidir=bool(rng.integers(0, 2)), in_dim=int(rng.integers(1, 120)), H=H,
+                          T=int(rng.integers(1, 6)), B=int(rng.integers(5, 33)), states=bool(rng.integers(0, 2)), seed=3000 + i))
+    return cases
+
+
+@pytest.mark.parametrize("c", _fuzz_batched(16, 77), ids=lambda c: "L{L}D{d}_in{in_dim}_H{H}_T{T}_B{B}".format(d=1 + c["bidir"], **c))
+def test_random_batched_shapes(oracle, c):
+    """Batches of 5 to 32 sequences at random widths: the batched tensor-core recurrence with and without
+    cluster pairs (odd CTA counts, slices too tall for a pair), its fall-backs (slice too large), and wide
+    bidirectional stacks whose directions run one after the other."""
+    scale = min(0.3, 2.0 / np.sqrt(c["H"] + c["in_dim"]))
+    w = wl.Workload("fuzzb", c["L"], c["bidir"], c["in_dim"], c["H"], c["T"], c["B"], "bf16", scale, seed=c["seed"])
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w) if c["states"] else (None, None)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got = run_gpu(w, weights, x, h0, c0)
+    assert_close(got, ref, "bf16", "fuzz batched")
