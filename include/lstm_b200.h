@@ -199,7 +199,8 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
  * [9] 1 if the recurrence keeps its weights in registers (bf16 dense), 0 for the shared-memory kernel,
  * [10] 16-column weight tiles per warp held in registers, [11] per warp held in shared memory,
  * [12] 1 if a call at max_B runs the batched tensor-core (tcgen05) recurrence: bf16 dense LSTM handles use
- * it for batches of 5 to 32 sequences and the register-resident kernel below that.
+ * it for batches of 5 to 64 sequences where its operand ring fits beside the resident slice, and the
+ * register-resident kernel (passes of four sequences) otherwise.
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 

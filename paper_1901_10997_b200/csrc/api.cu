@@ -630,7 +630,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     h->xch_words = (size_t)D * 2 * max_B * H;
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->xch, h->xch_words * 8, true, st, "exchange buffer");
     if (rc == LSTM_OK && h->use_tcb) {
-        rc = dev_alloc(h, &h->hplanes, (size_t)D * 2 * 64 * h->tcb_ldh * 2, true, st, "h planes");
+        rc = dev_alloc(h, &h->hplanes, (size_t)D * 2 * kTcPlaneRows * h->tcb_ldh * 2, true, st, "h planes");
         if (rc == LSTM_OK) rc = dev_alloc(h, &h->tcb_flags, (size_t)D * h->ncta_dir * sizeof(unsigned), true, st, "stamps");
     }
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
@@ -960,16 +960,20 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
             continue;
         }
-        if (h->use_tcb && B > 4 && B <= 32) {
+        int tc_kbs = 0, tc_stages = 0;
+        // the batched kernel serves this call if the operand ring for this batch fits beside the resident slice
+        // (the plan made at create time covers up to 32 sequences; larger batches may not fit and then run as
+        // passes of four on the kernels below)
+        if (h->use_tcb && B > 4 && B <= kTcMaxBatch &&
+            recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * B, 16), h->upc, B, (size_t)h->smem_optin - 256, h->tcb_pair ? 1 : 0, &tc_kbs, &tc_stages)) {
             RecurTcArgs m;
             memset(&m, 0, sizeof m);
             m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
             m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
             m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16);
             m.pair = h->tcb_pair ? 1 : 0;
-            if (!recur_tc_plan(m.RA, m.nkb, m.N, h->upc, B, (size_t)h->smem_optin - 256, m.pair, &m.kbs, &m.stages))
-                return fail(h, LSTM_ERR_INVALID, "batched recurrence does not fit shared memory at batch %d", B);
-            m.tmem_cols = m.N <= 32 ? 32 : 64;
+            m.kbs = tc_kbs; m.stages = tc_stages;
+            m.tmem_cols = m.N <= 32 ? 32 : m.N <= 64 ? 64 : 128;
             m.ldh = h->tcb_ldh;
             m.stamp_base = h->stamp_next;
             h->stamp_next += (unsigned)T + 1u;
@@ -1190,7 +1194,10 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
     }
     const Layer &l0 = h->layers[0];
     const int launches = h->last_launches > 0 ? h->last_launches : h->L * 2 + (h->use_tc ? 1 : 0);
-    const int tcb_at_max = (h->use_tcb && !h->Hh && h->max_B > 4 && h->max_B <= 32) ? 1 : 0;
+    int ik = 0, is = 0;
+    const int tcb_at_max = (h->use_tcb && !h->Hh && h->max_B > 4 && h->max_B <= kTcMaxBatch &&
+                            recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * h->max_B, 16), h->upc, h->max_B, (size_t)h->smem_optin - 256,
+                                          h->tcb_pair ? 1 : 0, &ik, &is)) ? 1 : 0;
     const int64_t vals[13] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->threads, (int64_t)shp.smem,
                               rows_res, rows_str, (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches,
                               h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0, tcb_at_max};

@@ -96,6 +96,8 @@ cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, siz
 // per 64 columns; h travels through global memory as bf16 planes [D][2 parities][64 rows][ldh] (row 2b = hi,
 // 2b+1 = lo part of batch row b) and one stamp per producer CTA.
 // ---------------------------------------------------------------------------------------------------
+constexpr int kTcMaxBatch = 64;       // sequences per call the batched tensor-core recurrence serves
+constexpr int kTcPlaneRows = 128;     // rows of one parity of the h planes: hi and lo row of every sequence
 struct RecurTcArgs {
     int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
     int H, B, T, D;

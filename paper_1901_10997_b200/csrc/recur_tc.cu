@@ -2,7 +2,7 @@
 // forward pass (paper, Section 4, cell equations with zero hidden layers per gate)
 //     z = G[t] + Wh h_{t-1};  i,f,o = sigmoid(z_i,z_f,z_o), g = tanh(z_g);  c_t = f c_{t-1} + i g;
 //     h_t = o tanh(c_t)
-// for batches of more than four sequences, where the per-step product Wh_slice [4u x H] . h_{t-1} [H x B]
+// for batches of five to kTcMaxBatch sequences, where the per-step product Wh_slice [4u x H] . h_{t-1} [H x B]
 // is a real (if skinny) matrix product and one tcgen05.mma chain per step replaces the ceil(B/4) passes of
 // the register-resident kernel.
 //
@@ -278,7 +278,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     volatile int *abort_flag = &abort_s;
     volatile int *pub = &pub_s;                 // steps this CTA has published (h0 counts as one)
 
-    __nv_bfloat16 *hbuf_d = a.hbuf + (size_t)d * 2 * 64 * a.ldh;            // [parity][64 rows][ldh]
+    __nv_bfloat16 *hbuf_d = a.hbuf + (size_t)d * 2 * kTcPlaneRows * a.ldh;  // [parity][kTcPlaneRows rows][ldh]
     unsigned *flags_d = a.flags + (size_t)d * a.ncta_dir;
 
     if (warp == 0) {
@@ -342,7 +342,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             if (aborted) break;
             fence_acq_rel_gpu();                                    // acquire: the planes behind the stamps
             asm volatile("fence.proxy.async;" ::: "memory");       // they were written with ordinary stores
-            const int row0 = (d * 2 + ((s + 1) & 1)) * 64;          // planes of step s-1 live in parity (s-1)&1
+            const int row0 = (d * 2 + ((s + 1) & 1)) * kTcPlaneRows;   // planes of step s-1 live in parity (s-1)&1
             for (int g0 = 0; g0 < nkb_my; g0 += kbs) {
                 const int nblk = min(kbs, nkb_my - g0);
                 int ok = 1;
@@ -404,7 +404,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             const int b = p / nu, u = p - b * nu;
             const float v = a.h0 ? a.h0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-            __nv_bfloat16 *row = hbuf_d + ((size_t)1 * 64 + 2 * b) * a.ldh + u0 + u;     // step -1 -> parity 1
+            __nv_bfloat16 *row = hbuf_d + ((size_t)1 * kTcPlaneRows + 2 * b) * a.ldh + u0 + u;     // step -1 -> parity 1
             row[0] = hi;
             row[a.ldh] = __float2bfloat16_rn(v - __bfloat162float(hi));
         }
@@ -442,25 +442,45 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             const bool mine = !pair || half == rank;
             const bool row_ok = row < RT && lr < 4 * (mine ? nu : nu_partner);
             if (lq * 32 < (pair ? RT : 4 * nu)) {
-                // all column chunks are requested before the one wait (N <= 64: at most four chunks of 16)
-                uint32_t v[4][16];
+                // the first four column chunks of 16 (all there are up to 32 sequences) are requested before
+                // one wait; batches above 32 read their remaining chunks one at a time (registers)
                 const int nchunk = (2 * B + 15) >> 4;
+                {
+                    uint32_t v[4][16];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (c < nchunk) tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(c * 16), v[c]);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row_ok) {
+                    for (int c = 0; c < 4; ++c)
+                        if (c < nchunk) tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(c * 16), v[c]);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (row_ok) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < nchunk) {
+                        for (int c = 0; c < 4; ++c) {
+                            if (c < nchunk) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                const int b = c * 8 + i;
-                                const float z = __uint_as_float(v[c][2 * i]) + __uint_as_float(v[c][2 * i + 1]);
-                                if (b < B) {
-                                    if (mine) zs[b * zld + lr] = z;
-                                    else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                                for (int i = 0; i < 8; ++i) {
+                                    const int b = c * 8 + i;
+                                    const float z = __uint_as_float(v[c][2 * i]) + __uint_as_float(v[c][2 * i + 1]);
+                                    if (b < B) {
+                                        if (mine) zs[b * zld + lr] = z;
+                                        else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                                    }
                                 }
+                            }
+                        }
+                    }
+                }
+#pragma unroll 1
+                for (int c = 4; c < nchunk; ++c) {
+                    uint32_t w[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(c * 16), w);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (row_ok) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int b = c * 8 + i;
+                            const float z = __uint_as_float(w[2 * i]) + __uint_as_float(w[2 * i + 1]);
+                            if (b < B) {
+                                if (mine) zs[b * zld + lr] = z;
+                                else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
                             }
                         }
                     }
@@ -473,7 +493,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                 if (ftid == 0) mbar_arrive_remote_release(partial_bar_remote);
                 if (!mbar_wait_cluster(smem_u32(&partial_bar), (uint32_t)s & 1u, abort_flag)) break;
             }
-            __nv_bfloat16 *hp = hbuf_d + (size_t)(s & 1) * 64 * a.ldh;
+            __nv_bfloat16 *hp = hbuf_d + (size_t)(s & 1) * kTcPlaneRows * a.ldh;
             for (int i = 0; ftid + 128 * i < nuB; ++i) {
                 const int p = ftid + 128 * i;
                 const int b = p / nu, u = p - b * nu, j = u0 + u;       // consecutive threads, consecutive units
@@ -610,7 +630,7 @@ bool recur_tc_encode_weights(void *map, const void *w, long long rows, int ld, i
 }
 bool recur_tc_encode_planes(void *map, const void *hbuf, int D, int H, int ldh, int N)
 {
-    return encode_2d(map, hbuf, (long long)D * 2 * 64, H, ldh, N);
+    return encode_2d(map, hbuf, (long long)D * 2 * kTcPlaneRows, H, ldh, N);
 }
 
 cudaError_t recur_tc_prepare(int max_smem)

@@ -214,7 +214,10 @@ TC_SHAPES = [
     small("tc_h129_b32", 1, False, 33, 129, 4, 32, "bf16"),         # the largest batch (N = 64), ragged K tail of one column
     small("tc_h1000_b17", 2, False, 64, 1000, 3, 17, "bf16", scale=0.05),   # 16 K blocks, four per stage; two layers
     small("tc_h1600_b9", 1, False, 32, 1600, 2, 9, "bf16", scale=0.03),     # 25 K blocks: the ring is down to a few stages
-    small("tc_h600_b32", 1, True, 24, 600, 3, 32, "bf16", scale=0.05),      # cluster pairs, both directions, largest batch
+    small("tc_h600_b32", 1, True, 24, 600, 3, 32, "bf16", scale=0.05),      # cluster pairs, both directions
+    small("tc_h300_b64", 2, True, 24, 300, 3, 64, "bf16", scale=0.05),      # the largest batch (N = 128): two rounds of accumulator chunks
+    small("tc_h1500_b48", 1, False, 40, 1500, 2, 48, "bf16", scale=0.03),   # N = 96 beside the full-width slice: two-block stages
+    small("tc_h1500_b64", 1, False, 40, 1500, 2, 64, "bf16", scale=0.03),   # N = 128 beside the full-width slice: one-block stages
     small("tc_h592_b6_t1", 1, False, 16, 592, 1, 6, "bf16", scale=0.05),    # cluster pairs, a single step, uneven K halves (10 blocks: 5 + 5; 592 = 9.25 blocks)
     # 14 units per CTA x 32 K blocks do not fit shared memory: the handle keeps the register-resident kernel
     small("notc_h2000_b9", 1, False, 32, 2000, 2, 9, "bf16", scale=0.03),
