@@ -76,12 +76,21 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4 &a, unsigned
 
 // gate functions from the fast exponential: absolute error of a few 1e-7, far inside the 2e-2 bound of
 // the bf16 storage type
-__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
-__device__ __forceinline__ float tanh_fast(float z)
+// Both gate functions as one expression, sc / (1 + 2^(-k log2(e) z)) + of: the logistic function with
+// (k, sc, of) = (1, 1, 0) and tanh z = 2 logistic(2z) - 1 with (2, 2, -1).  One exponential and one
+// reciprocal on the path from the summed pre-activation to the published h, and no select between two
+// evaluated functions.
+__device__ __forceinline__ float ex2_fast(float x)
 {
-    const float t = __expf(-2.0f * fabsf(z));
-    return copysignf(__fdividef(1.0f - t, 1.0f + t), z);
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
+__device__ __forceinline__ float gate_fast(float z, float neg_k_log2e, float sc, float of)
+{
+    return fmaf(sc, __fdividef(1.0f, 1.0f + ex2_fast(neg_k_log2e * z)), of);
+}
+__device__ __forceinline__ float tanh_fast(float z) { return gate_fast(z, -2.0f * 1.4426950408889634f, 2.0f, -1.0f); }
 
 __device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
 {
@@ -158,6 +167,8 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
     const int fpart = lane % P, fgrp = lane / P;    // fgrp = fb * 4 + fq
     const int fb = fgrp >> 2, fq = fgrp & 3;
     const bool fin_warp = warp < nu;
+    // gate function of this lane's gate (fq == 2: the cell candidate, tanh; else the logistic function)
+    const float act_k = (fq == 2 ? -2.0f : -1.0f) * 1.4426950408889634f, act_sc = fq == 2 ? 2.0f : 1.0f, act_of = fq == 2 ? -1.0f : 0.0f;
     const int frow = warp * 4 + fq;
 
     // Warps whose column range lies beyond H have nothing to poll and finish no unit: they leave now
@@ -353,7 +364,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                 }
                 for (int o = P >> 1; o >= 1; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
                 z += (g_cur.v[0] + g_cur.v[1]) + (g_cur.v[2] + g_cur.v[3]);
-                const float act = (fq == 2) ? tanh_fast(z) : sigmoid_fast(z);
+                const float act = gate_fast(z, act_k, act_sc, act_of);
                 const int qb = fb * 4 * P;                 // lane of gate i of this batch row
                 const float vi = __shfl_sync(0xffffffffu, act, qb);
                 const float vf = __shfl_sync(0xffffffffu, act, qb + P);
