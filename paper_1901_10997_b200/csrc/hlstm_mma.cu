@@ -52,12 +52,15 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4 &a, unsigned
         : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
-__device__ __forceinline__ float tanh_fast(float z)
+// logistic function and tanh z = 2 logistic(2z) - 1, each one exponential and one reciprocal
+__device__ __forceinline__ float ex2_fast(float x)
 {
-    const float t = __expf(-2.0f * fabsf(z));
-    return copysignf(__fdividef(1.0f - t, 1.0f + t), z);
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
+__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + ex2_fast(-1.4426950408889634f * z)); }
+__device__ __forceinline__ float tanh_fast(float z) { return fmaf(2.0f, __fdividef(1.0f, 1.0f + ex2_fast(-2.8853900817779268f * z)), -1.0f); }
 
 __device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
 {
@@ -304,7 +307,10 @@ __global__ void __launch_bounds__(NW * 32, 1) hlstm_mma_kernel(const HlstmArgs a
                 z += __shfl_xor_sync(0xffffffffu, z, 2);
                 z += __shfl_xor_sync(0xffffffffu, z, 1);
                 z += b_out;
-                const float act = (fq == 2) ? tanh_fast(z) : sigmoid_fast(z);
+                // one expression for both gate functions: logistic, or tanh z = 2 logistic(2z) - 1 for the candidate
+                const float act = fmaf(fq == 2 ? 2.0f : 1.0f,
+                                       __fdividef(1.0f, 1.0f + ex2_fast((fq == 2 ? -2.8853900817779268f : -1.4426950408889634f) * z)),
+                                       fq == 2 ? -1.0f : 0.0f);
                 const float vi = __shfl_sync(0xffffffffu, act, 0);
                 const float vf = __shfl_sync(0xffffffffu, act, 8);
                 const float vg = __shfl_sync(0xffffffffu, act, 16);

@@ -202,12 +202,15 @@ __device__ __forceinline__ void cluster_sync_all()
 }
 __device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
-__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
-__device__ __forceinline__ float tanh_fast(float z)
+// logistic function and tanh z = 2 logistic(2z) - 1, each one exponential and one reciprocal
+__device__ __forceinline__ float ex2_fast(float x)
 {
-    const float t = __expf(-2.0f * fabsf(z));
-    return copysignf(__fdividef(1.0f - t, 1.0f + t), z);
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
+__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + ex2_fast(-1.4426950408889634f * z)); }
+__device__ __forceinline__ float tanh_fast(float z) { return fmaf(2.0f, __fdividef(1.0f, 1.0f + ex2_fast(-2.8853900817779268f * z)), -1.0f); }
 __device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
 {
     const int base = H / nc, rem = H % nc;
