@@ -97,6 +97,12 @@ typedef struct {
  *   w[layers*(1+bidir)], exec_mode LSTM_DENSE | LSTM_CSR, 1 <= max_T, 1 <= max_B,
  *   cuda_stream: a cudaStream_t (NULL = default stream) used for the uploads.
  * Synchronises the stream before returning.  On failure *out is NULL.
+ * Environment switches read at create time (for measurements and tests; unset = the library chooses):
+ *   LSTM_B200_RECUR = simt  shared-memory recurrent kernel instead of the register-resident one (bf16 dense)
+ *                   = mma   no batched tensor-core recurrence (batches above four run as passes of four)
+ *                   = tc1   batched tensor-core recurrence without cluster pairs
+ *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
+ *   LSTM_B200_SPIN_LIMIT = <clock ticks>  bound of every device-side wait (default about two seconds)
  */
 LSTM_API int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir, int dtype,
                 const lstm_weights *w, int exec_mode, int max_T, int max_B, void *cuda_stream);
