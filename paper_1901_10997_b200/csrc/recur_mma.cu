@@ -106,7 +106,9 @@ constexpr int kChunk = 4;     // batch rows per pass: hi and lo parts fill the 8
 
 // MT: 16-row tiles per CTA (4 gate rows x units, padded); NKR: 16-column tiles per warp held in
 // registers; NW: warps per CTA.
-template <int MT, int NKR, int NW>
+// STAGED: the pass over several batch rows that lands the exchange words in shared memory (cp.async); kept
+// out of the single-row instantiation, whose registers are all spoken for.
+template <int MT, int NKR, int NW, bool STAGED>
 __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArgs a)
 {
     constexpr int NT = NW * 32;
@@ -227,7 +229,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                         Bw[dof + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
                     }
                 }
-            } else if (a.staged) {
+            } else if (STAGED) {
                 // Several batch rows: too many words per lane to hold in registers at once, and polling
                 // them in rounds would cost one L2 round trip per round.  All words of the pass are
                 // copied to shared memory asynchronously in one go (pairs of words, 16 bytes); pairs whose
@@ -404,32 +406,33 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 
 typedef void (*KernelFn)(const RecurMmaArgs);
 
-template <int MT, int NW>
+template <int MT, int NW, bool STAGED>
 KernelFn pick_nkr(int nkr)
 {
     switch (nkr) {
-        case 2: return recur_mma_kernel<MT, 2, NW>;
-        case 4: return recur_mma_kernel<MT, 4, NW>;
-        case 6: return recur_mma_kernel<MT, 6, NW>;
-        case 8: return recur_mma_kernel<MT, 8, NW>;
+        case 2: return recur_mma_kernel<MT, 2, NW, STAGED>;
+        case 4: return recur_mma_kernel<MT, 4, NW, STAGED>;
+        case 6: return recur_mma_kernel<MT, 6, NW, STAGED>;
+        case 8: return recur_mma_kernel<MT, 8, NW, STAGED>;
         default: return nullptr;
     }
 }
-template <int NW>
+template <int NW, bool STAGED>
 KernelFn pick_mt(int mt, int nkr)
 {
     switch (mt) {
-        case 1: return pick_nkr<1, NW>(nkr);
-        case 2: return pick_nkr<2, NW>(nkr);
-        case 3: return pick_nkr<3, NW>(nkr);
-        case 4: return pick_nkr<4, NW>(nkr);
+        case 1: return pick_nkr<1, NW, STAGED>(nkr);
+        case 2: return pick_nkr<2, NW, STAGED>(nkr);
+        case 3: return pick_nkr<3, NW, STAGED>(nkr);
+        case 4: return pick_nkr<4, NW, STAGED>(nkr);
         default: return nullptr;
     }
 }
-KernelFn pick(int mt, int nkr, int nw)
+KernelFn pick(int mt, int nkr, int nw, bool staged)
 {
     if (!recur_mma_shape_ok(mt, nkr, nw)) return nullptr;
-    return nw == 8 ? pick_mt<8>(mt, nkr) : pick_mt<16>(mt, nkr);
+    if (staged) return nw == 8 ? pick_mt<8, true>(mt, nkr) : pick_mt<16, true>(mt, nkr);
+    return nw == 8 ? pick_mt<8, false>(mt, nkr) : pick_mt<16, false>(mt, nkr);
 }
 
 }  // namespace
@@ -451,14 +454,18 @@ size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int 
 
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 {
-    KernelFn fn = pick(mt, nkr, nw);
-    if (!fn) return cudaErrorInvalidValue;
-    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    for (int staged = 0; staged < 2; ++staged) {
+        KernelFn fn = pick(mt, nkr, nw, staged != 0);
+        if (!fn) return cudaErrorInvalidValue;
+        const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st)
 {
-    KernelFn fn = pick(mt, nkr, nw);
+    KernelFn fn = pick(mt, nkr, nw, a.staged != 0);
     if (!fn) return cudaErrorInvalidValue;
     RecurMmaArgs copy = a;
     void *params[] = {&copy};
