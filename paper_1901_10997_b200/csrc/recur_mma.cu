@@ -108,7 +108,8 @@ constexpr int kChunk = 4;     // batch rows per pass: hi and lo parts fill the 8
 // registers; NW: warps per CTA.
 // STAGED: the pass over several batch rows that lands the exchange words in shared memory (cp.async); kept
 // out of the single-row instantiation, whose registers are all spoken for.
-template <int MT, int NKR, int NW, bool STAGED>
+// ONE: a single sequence (B = 1): the batch-row arithmetic folds away at compile time.
+template <int MT, int NKR, int NW, bool STAGED, bool ONE>
 __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArgs a)
 {
     constexpr int NT = NW * 32;
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tig = lane & 3;
-    const int H = a.H, B = a.B, T = a.T, D = a.D;
+    const int H = a.H, B = ONE ? 1 : a.B, T = a.T, D = a.D;
     const int d = a.dir0 + blockIdx.x / a.ncta_dir;
     const int cta = blockIdx.x % a.ncta_dir;
     int u0, nu;
@@ -406,33 +407,35 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 
 typedef void (*KernelFn)(const RecurMmaArgs);
 
-template <int MT, int NW, bool STAGED>
+template <int MT, int NW, bool STAGED, bool ONE>
 KernelFn pick_nkr(int nkr)
 {
     switch (nkr) {
-        case 2: return recur_mma_kernel<MT, 2, NW, STAGED>;
-        case 4: return recur_mma_kernel<MT, 4, NW, STAGED>;
-        case 6: return recur_mma_kernel<MT, 6, NW, STAGED>;
-        case 8: return recur_mma_kernel<MT, 8, NW, STAGED>;
+        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE>;
+        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE>;
+        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE>;
+        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE>;
         default: return nullptr;
     }
 }
-template <int NW, bool STAGED>
+template <int NW, bool STAGED, bool ONE>
 KernelFn pick_mt(int mt, int nkr)
 {
     switch (mt) {
-        case 1: return pick_nkr<1, NW, STAGED>(nkr);
-        case 2: return pick_nkr<2, NW, STAGED>(nkr);
-        case 3: return pick_nkr<3, NW, STAGED>(nkr);
-        case 4: return pick_nkr<4, NW, STAGED>(nkr);
+        case 1: return pick_nkr<1, NW, STAGED, ONE>(nkr);
+        case 2: return pick_nkr<2, NW, STAGED, ONE>(nkr);
+        case 3: return pick_nkr<3, NW, STAGED, ONE>(nkr);
+        case 4: return pick_nkr<4, NW, STAGED, ONE>(nkr);
         default: return nullptr;
     }
 }
-KernelFn pick(int mt, int nkr, int nw, bool staged)
+// variant 0: several rows polled from registers, 1: several rows staged in shared memory, 2: one sequence
+KernelFn pick(int mt, int nkr, int nw, int variant)
 {
     if (!recur_mma_shape_ok(mt, nkr, nw)) return nullptr;
-    if (staged) return nw == 8 ? pick_mt<8, true>(mt, nkr) : pick_mt<16, true>(mt, nkr);
-    return nw == 8 ? pick_mt<8, false>(mt, nkr) : pick_mt<16, false>(mt, nkr);
+    if (variant == 1) return nw == 8 ? pick_mt<8, true, false>(mt, nkr) : pick_mt<16, true, false>(mt, nkr);
+    if (variant == 2) return nw == 8 ? pick_mt<8, false, true>(mt, nkr) : pick_mt<16, false, true>(mt, nkr);
+    return nw == 8 ? pick_mt<8, false, false>(mt, nkr) : pick_mt<16, false, false>(mt, nkr);
 }
 
 }  // namespace
@@ -454,8 +457,8 @@ size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int 
 
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 {
-    for (int staged = 0; staged < 2; ++staged) {
-        KernelFn fn = pick(mt, nkr, nw, staged != 0);
+    for (int variant = 0; variant < 3; ++variant) {
+        KernelFn fn = pick(mt, nkr, nw, variant);
         if (!fn) return cudaErrorInvalidValue;
         const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
         if (e != cudaSuccess) return e;
@@ -465,7 +468,7 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st)
 {
-    KernelFn fn = pick(mt, nkr, nw, a.staged != 0);
+    KernelFn fn = pick(mt, nkr, nw, a.staged ? 1 : (a.B == 1 ? 2 : 0));
     if (!fn) return cudaErrorInvalidValue;
     RecurMmaArgs copy = a;
     void *params[] = {&copy};
