@@ -208,7 +208,8 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
     };
 
     int it = 0;
-#pragma unroll 1
+    // two steps per loop body where registers allow it: the buffer parities become constants
+#pragma unroll(ONE && MT * NKR <= 12 ? 2 : 1)
     for (int s = 0; s < T; ++s) {
         const int t = d ? (T - 1 - s) : s;
 #pragma unroll 1
