@@ -109,7 +109,8 @@ constexpr int kChunk = 4;     // batch rows per pass: hi and lo parts fill the 8
 // STAGED: the pass over several batch rows that lands the exchange words in shared memory (cp.async); kept
 // out of the single-row instantiation, whose registers are all spoken for.
 // ONE: a single sequence (B = 1): the batch-row arithmetic folds away at compile time.
-template <int MT, int NKR, int NW, bool STAGED, bool ONE>
+// POLL3: a lane polls three words per round instead of four (single sequence, at most 96 columns per warp).
+template <int MT, int NKR, int NW, bool STAGED, bool ONE, bool POLL3>
 __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArgs a)
 {
     constexpr int NT = NW * 32;
@@ -291,23 +292,24 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                 const unsigned want = a.stamp_base + (unsigned)s;            // stamp of step s-1
                 const unsigned long long *src = xch_d + ((size_t)((s - 1) & 1) * B + b0) * H;
                 long long t_start = 0;
-                for (int base = 0; base < nwords; base += 32 * kPoll) {
+                constexpr int KP = POLL3 ? 3 : kPoll;
+                for (int base = 0; base < nwords; base += 32 * KP) {
                     unsigned pending = 0;
-                    int soff[kPoll], doff[kPoll];
+                    int soff[KP], doff[KP];
 #pragma unroll
-                    for (int i = 0; i < kPoll; ++i) {
+                    for (int i = 0; i < KP; ++i) {
                         const int idx = base + lane + 32 * i;
                         if (word_offsets(idx, soff[i], doff[i]) && idx < nwords) pending |= 1u << i;
                     }
                     if (*abort_v) pending = 0;
                     int rounds = 0;
                     while (pending) {
-                        unsigned long long w[kPoll];
+                        unsigned long long w[KP];
 #pragma unroll
-                        for (int i = 0; i < kPoll; ++i)
+                        for (int i = 0; i < KP; ++i)
                             if (pending & (1u << i)) w[i] = ld_relaxed_u64(src + soff[i]);
 #pragma unroll
-                        for (int i = 0; i < kPoll; ++i)
+                        for (int i = 0; i < KP; ++i)
                             if ((pending & (1u << i)) && (unsigned)(w[i] >> 32) == want) {
                                 const float v = __uint_as_float((unsigned)w[i]);
                                 const __nv_bfloat16 hi = __float2bfloat16_rn(v);
@@ -408,35 +410,37 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 
 typedef void (*KernelFn)(const RecurMmaArgs);
 
-template <int MT, int NW, bool STAGED, bool ONE>
+template <int MT, int NW, bool STAGED, bool ONE, bool POLL3>
 KernelFn pick_nkr(int nkr)
 {
     switch (nkr) {
-        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE>;
-        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE>;
-        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE>;
-        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE>;
+        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE, POLL3>;
+        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE, POLL3>;
+        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE, POLL3>;
+        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE, (POLL3 && false)>;     // 128 columns per warp: four words
         default: return nullptr;
     }
 }
-template <int NW, bool STAGED, bool ONE>
+template <int NW, bool STAGED, bool ONE, bool POLL3>
 KernelFn pick_mt(int mt, int nkr)
 {
     switch (mt) {
-        case 1: return pick_nkr<1, NW, STAGED, ONE>(nkr);
-        case 2: return pick_nkr<2, NW, STAGED, ONE>(nkr);
-        case 3: return pick_nkr<3, NW, STAGED, ONE>(nkr);
-        case 4: return pick_nkr<4, NW, STAGED, ONE>(nkr);
+        case 1: return pick_nkr<1, NW, STAGED, ONE, POLL3>(nkr);
+        case 2: return pick_nkr<2, NW, STAGED, ONE, POLL3>(nkr);
+        case 3: return pick_nkr<3, NW, STAGED, ONE, POLL3>(nkr);
+        case 4: return pick_nkr<4, NW, STAGED, ONE, POLL3>(nkr);
         default: return nullptr;
     }
 }
-// variant 0: several rows polled from registers, 1: several rows staged in shared memory, 2: one sequence
+// variant 0: several rows polled from registers, 1: several rows staged in shared memory, 2: one sequence,
+// 3: one sequence with at most 96 columns per warp (three polled words per lane)
 KernelFn pick(int mt, int nkr, int nw, int variant)
 {
     if (!recur_mma_shape_ok(mt, nkr, nw)) return nullptr;
-    if (variant == 1) return nw == 8 ? pick_mt<8, true, false>(mt, nkr) : pick_mt<16, true, false>(mt, nkr);
-    if (variant == 2) return nw == 8 ? pick_mt<8, false, true>(mt, nkr) : pick_mt<16, false, true>(mt, nkr);
-    return nw == 8 ? pick_mt<8, false, false>(mt, nkr) : pick_mt<16, false, false>(mt, nkr);
+    if (variant == 1) return nw == 8 ? pick_mt<8, true, false, false>(mt, nkr) : pick_mt<16, true, false, false>(mt, nkr);
+    if (variant == 2) return nw == 8 ? pick_mt<8, false, true, false>(mt, nkr) : pick_mt<16, false, true, false>(mt, nkr);
+    if (variant == 3) return nw == 8 ? pick_mt<8, false, true, true>(mt, nkr) : pick_mt<16, false, true, true>(mt, nkr);
+    return nw == 8 ? pick_mt<8, false, false, false>(mt, nkr) : pick_mt<16, false, false, false>(mt, nkr);
 }
 
 }  // namespace
@@ -458,7 +462,7 @@ size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int 
 
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 {
-    for (int variant = 0; variant < 3; ++variant) {
+    for (int variant = 0; variant < 4; ++variant) {
         KernelFn fn = pick(mt, nkr, nw, variant);
         if (!fn) return cudaErrorInvalidValue;
         const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
@@ -469,7 +473,8 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st)
 {
-    KernelFn fn = pick(mt, nkr, nw, a.staged ? 1 : (a.B == 1 ? 2 : 0));
+    const int variant = a.staged ? 1 : a.B != 1 ? 0 : (nkr + a.nkw_smem) * 16 <= 96 ? 3 : 2;
+    KernelFn fn = pick(mt, nkr, nw, variant);
     if (!fn) return cudaErrorInvalidValue;
     RecurMmaArgs copy = a;
     void *params[] = {&copy};
