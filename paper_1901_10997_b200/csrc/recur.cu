@@ -190,7 +190,8 @@ __device__ __forceinline__ double gate_fn(double z, bool is_tanh) { return is_ta
 __device__ __forceinline__ float tanh_t(float c) { return tanhf(c); }
 __device__ __forceinline__ double tanh_t(double c) { return tanh(c); }
 
-template <bool BF16, int BT, bool CSR>
+// ONE: a single sequence (B = 1, BT = 1): the batch-row arithmetic folds away at compile time.
+template <bool BF16, int BT, bool CSR, bool ONE = false>
 __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
 {
     typedef typename Types<BF16>::W WT;
@@ -204,7 +205,7 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nthreads = blockDim.x, nwarps = nthreads >> 5;
-    const int H = a.H, Hs = a.Hs, B = a.B, T = a.T, D = a.D;
+    const int H = a.H, Hs = a.Hs, B = ONE ? 1 : a.B, T = a.T, D = a.D;
     const int d = a.dir0 + blockIdx.x / a.ncta_dir;
     const int cta = blockIdx.x % a.ncta_dir;
     int u0, nu;
@@ -408,7 +409,7 @@ cudaError_t launch_bt(const RecurArgs &a, int threads, size_t smem, cudaStream_t
 {
     const void *fn = nullptr;
     switch (a.BT) {
-        case 1: fn = (const void *)recur_kernel<BF16, 1, CSR>; break;
+        case 1: fn = a.B == 1 ? (const void *)recur_kernel<BF16, 1, CSR, true> : (const void *)recur_kernel<BF16, 1, CSR>; break;
         case 2: fn = (const void *)recur_kernel<BF16, 2, CSR>; break;
         case 4: fn = (const void *)recur_kernel<BF16, 4, CSR>; break;
         case 8: fn = (const void *)recur_kernel<BF16, 8, CSR>; break;
@@ -424,6 +425,8 @@ cudaError_t prepare_all(int max_smem)
 {
     cudaError_t e;
     e = cudaFuncSetAttribute(recur_kernel<BF16, 1, CSR>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(recur_kernel<BF16, 1, CSR, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(recur_kernel<BF16, 2, CSR>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (e != cudaSuccess) return e;
