@@ -45,7 +45,8 @@ typedef struct lstm_handle lstm_handle;      /* opaque, library-owned */
 
 /* storage / arithmetic type */
 enum {
-    LSTM_F32       = 0,   /* fp32 weights, fp32 activations and state, fp32 accumulation              */
+    LSTM_F32       = 0,   /* fp32 weights, activations, state and outputs; dot products and gate
+                             functions are evaluated in fp64 (fp32 sums miss the 1e-4 bound near zero)  */
     LSTM_BF16W_F32S = 1   /* weights rounded to bf16 (nearest-even) at create time; the input
                              projection feeds the tensor cores with each activation as two bf16
                              terms (hi + lo, about 16 mantissa bits); state, accumulation, gates and
@@ -249,7 +250,8 @@ LSTM_API int lstm_fold_input_affine(const float *wx, const float *b, int rows, i
  *   wx [4H, in_dim], wh [4H, H] row-major fp32 and b [4H] (or NULL = zeros), gate row blocks i,f,g,o;
  *   x [T,B,in_dim]; h0, c0 [B,H] or NULL (zeros); y [T,B,H]; hT, cT [B,H] or NULL (not wanted).
  * All are DEVICE pointers and are only read (wx, wh, b, x, h0, c0) or written (y, hT, cT) by this call.
- * The same cell equations as lstm_forward, fp32 accumulation; weights are read through L2 every step
+ * The same cell equations and arithmetic as a LSTM_F32 handle (fp64 sums and gate functions, fp32
+ * storage); weights are read through L2 every step
  * (nothing is packed or kept on-chip), so this path is slower than a handle.
  * Scratch: the per-step exchange words and a status word live in a fixed array inside the library
  * image (about 128 KiB of device memory on every GPU that loads the library, held until exit).

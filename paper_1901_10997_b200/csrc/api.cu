@@ -69,7 +69,7 @@ struct lstm_handle {
     float *ybuf[2] = {nullptr, nullptr};
     unsigned long long *xch = nullptr; size_t xch_words = 0;
     int *status_dev = nullptr;
-    unsigned stamp_next = 0;
+    unsigned stamp_next = 1;           // stamps start at 1: a cleared exchange word or flag (0) never matches or exceeds a wanted stamp
     long long spin_limit = 2000000000LL;
     long long spin_limit_default = 2000000000LL;
     int withhold_cta = -1;             // failure-path self-test (lstm_selftest_timeout)
@@ -96,6 +96,17 @@ int fail(lstm_handle *h, int code, const char *fmt, ...)
     va_end(ap);
     if (h) h->err = buf; else g_create_error = buf;
     return code;
+}
+
+// A handle is bound to the device that was current in lstm_create: launching with another device current
+// would run kernels there on this device's pointers.
+int check_device(lstm_handle *h)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "cudaGetDevice failed: %s", cudaGetErrorString(cudaGetLastError()));
+    if (dev != h->device)
+        return fail(h, LSTM_ERR_INVALID, "the handle belongs to device %d but device %d is current; nothing launched", h->device, dev);
+    return LSTM_OK;
 }
 
 inline uint16_t f32_to_bf16_rne(float f)
@@ -884,6 +895,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
     if (!h) return LSTM_ERR_INVALID;
     if (T < 0 || B < 0 || T > h->max_T || B > h->max_B)
         return fail(h, LSTM_ERR_INVALID, "T=%d B=%d outside [0,%d] x [0,%d]", T, B, h->max_T, h->max_B);
+    if (const int drc = check_device(h)) return drc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->last_stream = st;
     const int L = h->L, D = h->D, H = h->H;
@@ -915,7 +927,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (cudaMemsetAsync(h->xch, 0, h->xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->rxch && cudaMemsetAsync(h->rxch, 0, h->rxch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->tcb_flags && cudaMemsetAsync(h->tcb_flags, 0, (size_t)D * h->ncta_dir * sizeof(unsigned), st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
-        h->stamp_next = 0;
+        h->stamp_next = 1;
     }
 
     for (int l = 0; l < L; ++l) {
@@ -1070,6 +1082,7 @@ int lstm_input_projection(lstm_handle *h, const float *x, int T, int B, float *g
         return fail(h, LSTM_ERR_INVALID, "T=%d B=%d outside [0,%d] x [0,%d]", T, B, h->max_T, h->max_B);
     if (T == 0 || B == 0) return LSTM_OK;
     if (!x || !g) return fail(h, LSTM_ERR_INVALID, "x and g must not be NULL");
+    if (const int drc = check_device(h)) return drc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->last_stream = st;
     h->ev_used = 0;
@@ -1104,6 +1117,7 @@ int lstm_forward_host(lstm_handle *h, const float *x, int T, int B, const float 
     if (!h) return LSTM_ERR_INVALID;
     if (T < 0 || B < 0 || T > h->max_T || B > h->max_B)
         return fail(h, LSTM_ERR_INVALID, "T=%d B=%d outside [0,%d] x [0,%d]", T, B, h->max_T, h->max_B);
+    if (const int drc = check_device(h)) return drc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t Mmax = (size_t)h->max_T * h->max_B;
     const size_t smax = (size_t)h->L * h->D * h->max_B * h->H;

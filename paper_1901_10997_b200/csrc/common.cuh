@@ -69,6 +69,7 @@ struct RecurMmaArgs {
     unsigned stamp_base;
     long long spin_limit;
     int withhold_cta;           // failure-path self-test: this CTA never publishes its h values (-1: none)
+    int probe;                  // measurement only (kProbe* bits): parts of a step left out, outputs undefined
     // per direction [cta][warp][column tile][row tile][lane] 16-byte operand-A fragments:
     // lane (g = lane / 4, p = lane % 4) holds rows g and g + 8, columns 2p, 2p+1 and 2p+8, 2p+9
     const uint4 *wfrag[2];
@@ -83,6 +84,10 @@ struct RecurMmaArgs {
     unsigned long long *xch;
     int *status;
 };
+// probe bits of the register-resident kernels: what a step leaves out when its cost is being measured
+constexpr int kProbeNoProducts = 1;   // no tensor instructions (partial sums are written as zeros)
+constexpr int kProbeNoGates = 2;      // no reduction, gate functions or output stores: the unit's word is published as it is
+constexpr int kProbeNoExchange = 4;   // no wait for the other CTAs' words
 constexpr int kMmaTileCap16 = 18;   // MT * NKR limit with 16 warps (128 registers per thread, no spills)
 constexpr int kMmaTileCap8 = 40;    // ... with 8 warps
 bool recur_mma_shape_ok(int mt, int nkr, int nw);

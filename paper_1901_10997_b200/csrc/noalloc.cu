@@ -9,7 +9,8 @@
 //
 // The kernel is a plain variant of the library's persistent recurrent kernel: weights stay in the
 // caller's row-major fp32 arrays and are read through L2 each step (nothing is packed or made
-// resident), the input half of the product is computed inside the step, accumulation is fp32.
+// resident), the input half of the product is computed inside the step; sums and gate functions are
+// evaluated in fp64 and stored as fp32, as in the handle's fp32 storage type.
 #include "../../include/lstm_b200.h"
 
 #include <cuda_runtime.h>
@@ -61,7 +62,6 @@ __global__ void __launch_bounds__(kThreads, 1) recur_noalloc_kernel(const Args a
     const int c = blockIdx.x;
     const int nu = base + (c < rem ? 1 : 0);
     const int u0 = c * base + (c < rem ? c : rem);
-    const int upc = base + (rem ? 1 : 0);
     const int V = in + H;                              // one staged row: [x_t | h_{t-1}]
     float *v_s = smem;                                 // [B][V]
     float *c_s = smem + (size_t)B * V;                 // [upc][B]
@@ -71,7 +71,6 @@ __global__ void __launch_bounds__(kThreads, 1) recur_noalloc_kernel(const Args a
         const int u = i / B, bb = i - u * B;
         c_s[u * B + bb] = a.c0 ? a.c0[(size_t)bb * H + u0 + u] : 0.0f;
     }
-    (void)upc;
     if (tid == 0) abort_s = 0;
     __syncthreads();
 
@@ -115,14 +114,16 @@ __global__ void __launch_bounds__(kThreads, 1) recur_noalloc_kernel(const Args a
             const int u = ub / B, bb = ub - u * B;
             const int j = u0 + u;
             const float *v = v_s + (size_t)bb * V;
-            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            // dot products and gate functions in fp64, like the handle's fp32 storage type: fp32 sums of a
+            // few hundred terms already miss the 1e-4 agreement bound on outputs near zero
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const float *rx = a.wx + (size_t)(q * H + j) * in;
                 const float *rh = a.wh + (size_t)(q * H + j) * H;
-                float sum = 0.0f;
-                for (int k = lane; k < in; k += 32) sum = fmaf(rx[k], v[k], sum);
-                for (int k = lane; k < H; k += 32) sum = fmaf(rh[k], v[in + k], sum);
+                double sum = 0.0;
+                for (int k = lane; k < in; k += 32) sum = fma((double)rx[k], (double)v[k], sum);
+                for (int k = lane; k < H; k += 32) sum = fma((double)rh[k], (double)v[in + k], sum);
                 acc[q] = sum;
             }
 #pragma unroll
@@ -130,16 +131,17 @@ __global__ void __launch_bounds__(kThreads, 1) recur_noalloc_kernel(const Args a
 #pragma unroll
                 for (int o = 16; o >= 1; o >>= 1) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
             if (lane == 0) {
-                const float zi = acc[0] + (a.b ? a.b[j] : 0.0f);
-                const float zf = acc[1] + (a.b ? a.b[H + j] : 0.0f);
-                const float zg = acc[2] + (a.b ? a.b[2 * H + j] : 0.0f);
-                const float zo = acc[3] + (a.b ? a.b[3 * H + j] : 0.0f);
-                const float gi = 1.0f / (1.0f + expf(-zi));
-                const float gf = 1.0f / (1.0f + expf(-zf));
-                const float gg = tanhf(zg);
-                const float go = 1.0f / (1.0f + expf(-zo));
-                const float cn = fmaf(gf, c_s[u * B + bb], gi * gg);
-                const float hn = go * tanhf(cn);
+                const double zi = acc[0] + (a.b ? (double)a.b[j] : 0.0);
+                const double zf = acc[1] + (a.b ? (double)a.b[H + j] : 0.0);
+                const double zg = acc[2] + (a.b ? (double)a.b[2 * H + j] : 0.0);
+                const double zo = acc[3] + (a.b ? (double)a.b[3 * H + j] : 0.0);
+                const double gi = 1.0 / (1.0 + exp(-zi));
+                const double gf = 1.0 / (1.0 + exp(-zf));
+                const double gg = tanh(zg);
+                const double go = 1.0 / (1.0 + exp(-zo));
+                const double cn_d = fma(gf, (double)c_s[u * B + bb], gi * gg);
+                const float cn = (float)cn_d;
+                const float hn = (float)(go * tanh(cn_d));
                 c_s[u * B + bb] = cn;
                 st_relaxed_u64(&sc->xch[s & 1][(size_t)bb * H + j],
                                ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned long long)__float_as_uint(hn));

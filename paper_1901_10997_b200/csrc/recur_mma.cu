@@ -232,6 +232,8 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                         Bw[dof + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
                     }
                 }
+            } else if (a.probe & kProbeNoExchange) {
+                // measurement only: no wait for the other CTAs, the operand keeps whatever it holds
             } else if (STAGED) {
                 // Several batch rows: too many words per lane to hold in registers at once, and polling
                 // them in rounds would cost one L2 round trip per round.  All words of the pass are
@@ -338,18 +340,20 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
             for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
+            if (!(a.probe & kProbeNoProducts)) {
 #pragma unroll
-            for (int i = 0; i < NKR; ++i) {
-                const unsigned bv0 = Bw32[i * 64 + g * 8 + tig];
-                const unsigned bv1 = Bw32[i * 64 + g * 8 + tig + 4];
+                for (int i = 0; i < NKR; ++i) {
+                    const unsigned bv0 = Bw32[i * 64 + g * 8 + tig];
+                    const unsigned bv1 = Bw32[i * 64 + g * 8 + tig + 4];
 #pragma unroll
-                for (int mt = 0; mt < MT; ++mt) mma_bf16(acc[mt], areg[i][mt], bv0, bv1);
-            }
-            for (int i = 0; i < nks; ++i) {
-                const unsigned bv0 = Bw32[(NKR + i) * 64 + g * 8 + tig];
-                const unsigned bv1 = Bw32[(NKR + i) * 64 + g * 8 + tig + 4];
+                    for (int mt = 0; mt < MT; ++mt) mma_bf16(acc[mt], areg[i][mt], bv0, bv1);
+                }
+                for (int i = 0; i < nks; ++i) {
+                    const unsigned bv0 = Bw32[(NKR + i) * 64 + g * 8 + tig];
+                    const unsigned bv1 = Bw32[(NKR + i) * 64 + g * 8 + tig + 4];
 #pragma unroll
-                for (int mt = 0; mt < MT; ++mt) mma_bf16(acc[mt], As_w[(size_t)(i * MT + mt) * 32], bv0, bv1);
+                    for (int mt = 0; mt < MT; ++mt) mma_bf16(acc[mt], As_w[(size_t)(i * MT + mt) * 32], bv0, bv1);
+                }
             }
             // accumulator columns 2*tig and 2*tig+1 are the hi and lo parts of batch row tig
             float *rw = red + (size_t)((it & 1) * NW + warp) * WS + tig * RP + g;
@@ -362,7 +366,12 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
             // ---- all partial sums of this pass are in place (two barriers and two buffers alternate)
             bar_sync(1 + (it & 1), nbar);
 
-            if (fin_warp) {
+            if (fin_warp && (a.probe & kProbeNoGates)) {
+                // measurement only: the exchange without the reduction, the gate functions and the outputs
+                if (fq == 0 && fpart == 0 && fb < nb && (int)blockIdx.x != a.withhold_cta)
+                    st_relaxed_u64(xch_d + ((size_t)(s & 1) * B + b0 + fb) * H + u0 + warp,
+                                   ((unsigned long long)(a.stamp_base + (unsigned)s + 1u) << 32) | 0x3e800000ull);
+            } else if (fin_warp) {
                 float z = 0.0f;
                 if (fb < nb) {
                     const float *rp = red + (size_t)((it & 1) * NW) * WS + fb * RP + frow;

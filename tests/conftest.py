@@ -33,3 +33,19 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """With LSTM_B200_ERRLOG=<file>, writes every (case, tensor, storage type, floored, scaled) error the GPU
+    parity helpers measured in this session, one JSON record per line."""
+    path = os.environ.get("LSTM_B200_ERRLOG")
+    if not path:
+        return
+    try:
+        import json
+        import gpu_util
+        with open(path, "w") as f:
+            for rec in gpu_util.ERR_LOG:
+                f.write(json.dumps(rec) + "\n")
+    except Exception:
+        pass

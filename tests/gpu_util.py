@@ -43,8 +43,20 @@ def run_gpu(w: wl.Workload, weights, x, h0=None, c0=None, exec_mode="dense", max
         m.close()
 
 
-def assert_close(got, ref, dtype, what=""):
+# Regression guard beside the contract tolerance: the SCALED error (max |diff| / max |ref|) must stay within a
+# few times of what the kernels deliver today, so that a lost low-order activation plane or a dropped
+# partial sum fails a test although it would still fit the contract tolerance.  Set from measured runs
+# (every recorded case, largest value per storage type, times three).
+GUARD = {"fp32": 3.5e-7, "bf16": 7e-5}      # measured maxima over the whole suite: 1.07e-7 and 2.37e-5
+
+ERR_LOG = []      # (what, tensor, dtype, floored, scaled) of every comparison, written out by conftest on request
+
+
+def assert_close(got, ref, dtype, what="", guard=None):
     tol = wl.TOLERANCE[dtype]
+    guard = GUARD[dtype] if guard is None else guard
     for name, g, r in zip(("y", "hT", "cT"), got, ref):
         floored, scaled = wl.rel_err(g, r)
+        ERR_LOG.append((what, name, dtype, floored, scaled))
         assert floored <= tol, f"{what} {name}: floored rel err {floored:.3e} (scaled {scaled:.3e}) > {tol}"
+        assert scaled <= guard, f"{what} {name}: scaled err {scaled:.3e} above the regression guard {guard:.1e} (floored {floored:.3e})"

@@ -1,4 +1,4 @@
-"""lstm_forward_noalloc against lstm_forward (needs a B200).
+"""lstm_forward_noalloc against lstm_forward and against the fp64 oracle (needs a B200).
 
 The entry point under test serves callers that are not allowed to allocate device memory when they
 run the model (fixed memory pools, an allocator owned by someone else): it works straight from the
@@ -41,7 +41,7 @@ def _noalloc_path(pkg, torch, w, weights, x, h0, c0):
     return y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()
 
 
-def test_two_calls_in_a_row_match_the_handle_path():
+def test_two_calls_in_a_row_match_the_handle_path(oracle):
     import torch
     import paper_1901_10997_b200 as pkg
     tol = wl.TOLERANCE["fp32"]
@@ -55,6 +55,11 @@ def test_two_calls_in_a_row_match_the_handle_path():
         for name, g, r in zip(("y", "hT", "cT"), got, want):
             floored, scaled = wl.rel_err(g, r)
             assert floored <= tol, f"{w.name} {name}: {floored:.3e} (scaled {scaled:.3e}) > {tol}"
+        # and against the independent CPU oracle, so that the two CUDA paths cannot be wrong together
+        ref = oracle.forward(weights, x, h0, c0, layers=1, bidir=False, hidden=w.hidden)
+        for name, g, r in zip(("y", "hT", "cT"), got, (ref[0], ref[1][0], ref[2][0])):
+            floored, scaled = wl.rel_err(g, r)
+            assert floored <= tol, f"{w.name} {name} vs oracle: {floored:.3e} (scaled {scaled:.3e}) > {tol}"
 
 
 def test_sizes_beyond_the_built_in_scratch_are_rejected():
