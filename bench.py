@@ -6,23 +6,32 @@ Default run (one JSON line on stdout):
 A step is one lstm_forward over the large language-model workload (2 layers, 1500 -> 1500, T = 35,
 batch 1, bf16 weights / fp32 state): input projection for all timesteps + serial recurrence, every
 layer.  `value` is microseconds per sequence with inputs resident in device memory; `e2e` is the same
-through lstm_forward_host with pinned host buffers (copies inside the timed region).  With N > 1 each
-rank runs an independent replica (batch columns and sequences never interact): no collective on the
-data path, N sequences per step.
+through lstm_forward_host with pinned host buffers (copies inside the timed region).  At one GPU the
+line also carries short device-timed `legs` for the other workloads (batches of 20 and 16 sequences, the
+pruned stack dense-with-zeros against CSR, the speech-shaped stack, the small fp32 stack), the on-chip
+yardstick of the recurrent step (`roofline.on_chip`: the exchange-only step measured by the library's own
+probe modes) and the fp64 CPU oracle timed on the host cores (all threads and one thread).
+With N > 1 each rank runs an independent replica (batch columns and sequences never interact): no
+collective on the data path, N sequences per step.  Started without a launcher, `--gpus N` starts the N
+ranks itself (one process per GPU, rendezvous on 127.0.0.1).
 
 Other modes:
     --impl reference     time the fp64 CPU oracle on the same workload (host cores only)
     --sweep              latency vs hidden size (H = 128..2048 step 8) with the LHP analysis
     --matmul-sweep       dense (tensor-core) vs sparse (CSR) matrix product at batch 16, d = 128..2048
     --workload NAME      cfg1 | cfg2 | cfg2_b20 | cfg4_10 | cfg4_05 | cfg4_10_csr | cfg4_05_csr |
-                         cfg5 | cfg5_b16 (default cfg2)
+                         cfg5 | cfg5_b16 | hlstm_ptb | hlstm_ds2 (default cfg2)
+    --no-legs            headline workload only
+    --out DIR            where the sweeps write their tables (default bench_out)
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -36,6 +45,12 @@ sys.path.insert(0, str(ROOT))
 import lstm_workloads as wl  # noqa: E402
 
 FALLBACK_HBM_GBS = 6650.0
+
+# legs of the default line at one GPU: (key, --workload name, timed steps)
+LEGS = [("cfg2_b20", "cfg2_b20", 20), ("cfg5_b16", "cfg5_b16", 3), ("cfg5_b1", "cfg5", 5),
+        ("cfg4_d10_dense_with_zeros", "cfg4_10", 20), ("cfg4_d10_csr", "cfg4_10_csr", 20),
+        ("cfg4_d05_dense_with_zeros", "cfg4_05", 20), ("cfg4_d05_csr", "cfg4_05_csr", 20),
+        ("cfg1_fp32_b20", "cfg1", 20)]
 
 
 def pick_workload(name: str):
@@ -69,21 +84,23 @@ def measured_peaks():
 
 
 def measured_traffic(kernel: str, workload: str, source: str):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary
-    profiles/<kernel>_<workload>.md, or None when there is none or the kernel's source has changed since
-    the counters were taken (the summary records the sha256 of the source file it profiled)."""
+    """(DRAM bytes per launch, where they come from) of the dominant kernel from the committed ncu summary
+    profiles/<kernel>_<workload>.md; (None, reason) when there is none or the kernel's source has changed
+    since the counters were taken (the summary records the sha256 of the source file it profiled)."""
     import hashlib
     import re
     f = ROOT / "profiles" / f"{kernel}_{workload}.md"
     src = ROOT / "paper_1901_10997_b200" / "csrc" / source
     if not (f.exists() and src.exists()):
-        return None
+        return None, "no ncu summary for this kernel and workload"
     text = f.read_text()
     m_sha = re.search(r"source_sha256:\s*([0-9a-f]{64})", text)
     m_tr = re.search(r"traffic_bytes_per_launch:\s*([0-9]+)", text)
-    if not (m_sha and m_tr) or hashlib.sha256(src.read_bytes()).hexdigest() != m_sha.group(1):
-        return None
-    return int(m_tr.group(1))
+    if not (m_sha and m_tr):
+        return None, f"profiles/{f.name} carries no counters"
+    if hashlib.sha256(src.read_bytes()).hexdigest() != m_sha.group(1):
+        return None, f"profiles/{f.name} was taken from an earlier revision of {source}"
+    return int(m_tr.group(1)), f"profiles/{f.name} (one ncu capture, dram__bytes_read.sum + dram__bytes_write.sum; not measured in this run)"
 
 
 def make_inputs(w: wl.Workload, mode: str):
@@ -147,7 +164,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.01)
+            self._stop.wait(0.005)
 
     def __enter__(self):
         if self._nv is not None:
@@ -181,28 +198,67 @@ def oracle_time(w: wl.Workload, weights, x, target_seconds=12.0, max_reps=400, m
     return per_seq, reps, oracle.threads()
 
 
+def oracle_time_one_thread(workload: str, reps: int = 3):
+    """The same oracle on ONE host thread: a child process started with OMP_NUM_THREADS=1 (the thread count of
+    an OpenMP library is fixed when it loads), whole sequences of the workload, one batch column.  Returns
+    microseconds per sequence, or None if the child failed."""
+    code = ("import sys, time, json; sys.path.insert(0, %r); import bench; "
+            "w, mode = bench.pick_workload(%r); weights, x = bench.make_inputs(w, mode); xs = x[:, :1]; "
+            "bench.oracle_forward(w, mode, weights, xs); t0 = time.perf_counter(); "
+            "[bench.oracle_forward(w, mode, weights, xs) for _ in range(%d)]; "
+            "import oracle; print(json.dumps({'us': (time.perf_counter() - t0) / %d * 1e6, 'threads': oracle.threads()}))"
+            % (str(ROOT), workload, reps, reps))
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    try:
+        r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+        d = json.loads(r.stdout.strip().splitlines()[-1])
+        return float(d["us"]) if int(d["threads"]) == 1 else None
+    except Exception:
+        return None
+
+
+def workload_config(w: wl.Workload, mode: str, world: int = 1):
+    return {"workload": w.name, "layers": w.layers, "dirs": w.dirs, "in_dim": w.in_dim, "hidden": w.hidden,
+            "T": w.T, "B": w.B, "exec_mode": mode, "weights": w.dtype, "state": "fp32",
+            "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world}"}
+
+
 def run_reference(args):
+    """The reference arm: the fp64 oracle as it stands on the host cores, same workload and metric.  A step is
+    one whole sequence (one batch column) of the workload.  --steps / --warmup are honoured unless the run
+    would pass three minutes, in which case fewer steps are timed and the line says how many."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w, _mode = pick_workload(args.workload)
-    weights, x = make_inputs(w, _mode)
+    w, mode = pick_workload(args.workload)
+    weights, x = make_inputs(w, mode)
     import oracle
     xs = x[:, :1] if w.B > 1 else x
-    for _ in range(min(args.warmup, 1)):
-        oracle_forward(w, _mode, weights, xs)
-    steps = max(1, min(args.steps, 10))
+    budget = 180.0
+    t_begin = time.perf_counter()
+    t0 = time.perf_counter()
+    oracle_forward(w, mode, weights, xs)
+    first = time.perf_counter() - t0
+    warm = max(0, args.warmup - 1)
+    warm = int(min(warm, max(0, (0.25 * budget - first) / max(first, 1e-9))))
+    for _ in range(warm):
+        oracle_forward(w, mode, weights, xs)
+    left = budget - (time.perf_counter() - t_begin)
+    steps = int(max(1, min(args.steps, left / max(first, 1e-9))))
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle_forward(w, _mode, weights, xs)
+        oracle_forward(w, mode, weights, xs)
     per_seq = (time.perf_counter() - t0) / steps
     us = per_seq * 1e6
     sample = f"{steps} whole sequences of {w.name} (T={w.T}, one batch column per step), fp64 oracle"
+    cfg = workload_config(w, mode, 1)
+    cfg["l2"] = "not applicable (host)"
+    cfg["parallelism"] = "host threads (OpenMP over independent outputs)"
     print(json.dumps({
         "impl": "reference", "metric": "us_per_sequence", "value": us, "unit": "us", "n_gpus": args.gpus,
-        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": per_seq * 1e3, "higher_is_better": False,
+        "steps": steps, "warmup": min(args.warmup, warm + 1), "ms_per_step": per_seq * 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "layers": w.layers, "hidden": w.hidden, "T": w.T, "B": 1},
+        "config": cfg,
         "cpu_baseline": {"value": us, "unit": "us", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -248,6 +304,156 @@ def time_steps(fn, steps, warmup, flush_buf, torch):
     return [s.elapsed_time(e) for s, e in zip(starts, ends)]
 
 
+def time_back_to_back(fn, calls, reps, torch):
+    """`calls` calls inside ONE event pair, `reps` pairs: the per-call time no longer depends on the tick of the
+    event clock; L2 stays warm (the serving-loop case).  Returns the median per-call milliseconds."""
+    fn()
+    torch.cuda.synchronize()
+    out = []
+    for _ in range(reps):
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(calls):
+            fn()
+        e.record()
+        torch.cuda.synchronize()
+        out.append(s.elapsed_time(e) / calls)
+    return float(np.median(out))
+
+
+def trimmed_mean(ms, drop=0.1):
+    """Mean without the slowest `drop` share of the samples: unlike a median it resolves differences below the
+    tick of the event clock (the ticks average out over the samples)."""
+    v = sorted(ms)
+    keep = v[:max(1, int(round(len(v) * (1.0 - drop))))]
+    return float(sum(keep) / len(keep))
+
+
+def kernel_of(info, mode):
+    if mode == "hlstm":
+        return "hlstm_mma_kernel", "hlstm_mma.cu"
+    if mode == "csr":
+        return ("recur_csr_kernel", "recur_csr.cu") if info.get("recur_register_resident") else ("recur_kernel", "recur.cu")
+    if info.get("recur_batched_tensor_core"):
+        return "recur_tc_kernel", "recur_tc.cu"
+    if info.get("recur_register_resident"):
+        return "recur_mma_kernel", "recur_mma.cu"
+    return "recur_kernel", "recur.cu"
+
+
+class GpuCase:
+    """One workload on one device: handle, device buffers, and the timed regions."""
+
+    def __init__(self, torch, pkg, workload_name, dev, flush_buf, weights_cache=None):
+        self.torch, self.pkg = torch, pkg
+        self.name = workload_name
+        self.w, self.mode = pick_workload(workload_name)
+        w = self.w
+        key = (w.seed, w.layers, w.bidir, w.in_dim, w.hidden, w.dtype, w.density, self.mode == "hlstm")
+        if weights_cache is not None and key in weights_cache and weights_cache[key][1].shape[1] >= w.B:
+            self.weights, xs = weights_cache[key]
+            self.x = np.ascontiguousarray(xs[:, :w.B])
+        else:
+            self.weights, self.x = make_inputs(w, self.mode)
+            if weights_cache is not None:
+                weights_cache[key] = (self.weights, self.x)
+        if self.mode == "hlstm":
+            self.model = pkg.HLSTM(self.weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, gate_hidden=w.hidden,
+                                   bidir=w.bidir, dtype=w.dtype, max_T=w.T, max_B=w.B)
+        else:
+            self.model = pkg.LSTM(self.weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir,
+                                  dtype=w.dtype, exec_mode=self.mode, max_T=w.T, max_B=w.B)
+        self.dev = dev
+        self.flush_buf = flush_buf
+        self.xd = torch.from_numpy(self.x).to(dev)
+        self.out = (torch.empty((w.T, w.B, w.dirs * w.hidden), device=dev),
+                    torch.empty((w.layers * w.dirs, w.B, w.hidden), device=dev),
+                    torch.empty((w.layers * w.dirs, w.B, w.hidden), device=dev))
+
+    def step(self):
+        self.model.forward(self.xd, out=self.out)
+
+    def timed(self, steps, warmup):
+        ms = time_steps(self.step, steps, warmup, self.flush_buf, self.torch)
+        self.model.check()
+        return ms
+
+    def kernel_split(self, steps, warmup=3):
+        """The same region again with the library's per-kernel events: (recurrence ms, recurrence launches,
+        projection ms, staging ms), totals over `steps` forwards."""
+        pkg, m = self.pkg, self.model
+        m.profile_enable(True)
+        rec_ms, rec_n, proj_ms, stage_ms = 0.0, 0, 0.0, 0.0
+        for i in range(steps + warmup):
+            flush_l2(self.flush_buf)
+            self.step()
+            n, t = m.profile_read()
+            if i >= warmup:
+                rec_ms += t[pkg.LSTM_K_RECUR]; rec_n += n[pkg.LSTM_K_RECUR]
+                proj_ms += t[pkg.LSTM_K_PROJ]; stage_ms += t[pkg.LSTM_K_STAGE]
+        m.profile_enable(False)
+        return rec_ms, rec_n, proj_ms, stage_ms
+
+    def nnz(self):
+        if self.mode != "csr":
+            return None
+        w = self.w
+        return float(np.mean([sum(int(np.count_nonzero(self.weights[l * w.dirs + d]["mask_h"])) for d in range(w.dirs))
+                              for l in range(w.layers)]))
+
+    def roofline(self, rec_ms, rec_n, peak, peak_kind):
+        w = self.w
+        alg_bytes = recurrence_bytes_per_launch(w, "hlstm" if self.mode == "hlstm" else self.nnz())
+        rec_avg_ms = rec_ms / max(rec_n, 1)
+        achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
+        info = self.model.info()
+        kernel_name, kernel_src = kernel_of(info, self.mode)
+        traffic, source = measured_traffic(kernel_name, self.name, kernel_src)
+        steps_per_launch = w.T * (2 if (w.dirs == 2 and info.get("ctas_per_dir") == info.get("sm_count")) else 1)
+        return {"bound": "hbm", "kernel": f"{kernel_name} (one launch = one layer, all T steps)",
+                "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": (achieved / peak if achieved else None), "peak_kind": f"of {peak_kind}",
+                "traffic": traffic, "traffic_source": source, "algorithmic_bytes_per_launch": alg_bytes,
+                "avg_launch_ms": rec_avg_ms, "us_per_timestep": rec_avg_ms * 1e3 / steps_per_launch,
+                "note": "the recurrent matrix stays on-chip (registers / shared memory) for the whole sequence, so the "
+                        "fraction of the per-step HBM weight-read bound may exceed 1; on_chip holds the bound that binds"}
+
+    def on_chip(self, steps):
+        """The yardstick that binds once the matrix is on-chip: the dependency chain of one step.  Uses the
+        library's probe modes (parts of the step left out) on this very handle and workload; every figure is the
+        recurrent kernel's launch time / T, prologue included."""
+        pkg, m, w = self.pkg, self.model, self.w
+        try:
+            m.probe(0)
+        except pkg.LstmError:
+            return None
+        res = {}
+        modes = [("step_us", 0),
+                 ("empty_step_us", pkg.LSTM_PROBE_NO_PRODUCTS | pkg.LSTM_PROBE_NO_GATES),
+                 ("exchange_and_gates_us", pkg.LSTM_PROBE_NO_PRODUCTS),
+                 ("compute_only_us", pkg.LSTM_PROBE_NO_EXCHANGE),
+                 ("products_only_us", pkg.LSTM_PROBE_NO_EXCHANGE | pkg.LSTM_PROBE_NO_GATES)]
+        try:
+            for key, mask in modes:
+                m.probe(mask)
+                rec_ms, rec_n, _p, _s = self.kernel_split(steps)
+                m.check()
+                res[key] = rec_ms / max(rec_n, 1) * 1e3 / w.T
+        finally:
+            m.probe(0)
+        self.step()                 # leave valid outputs behind
+        m.check()
+        res["step_over_empty_step"] = res["step_us"] / res["empty_step_us"] if res.get("empty_step_us") else None
+        res["what"] = ("per timestep, measured by the library (lstm_probe): empty_step = publish -> L2 -> poll + CTA barrier, "
+                       "no products, no gate functions; compute_only = products + barrier + reduction + gates + stores without "
+                       "waiting for other CTAs; the weights are read from the register file, so no shared-memory or HBM "
+                       "bandwidth bounds the step: the exchange latency does")
+        return res
+
+    def close(self):
+        self.model.close()
+
+
 def run_gpu(args):
     import torch
     import paper_1901_10997_b200 as pkg
@@ -256,13 +462,19 @@ def run_gpu(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     w, mode = pick_workload(args.workload)
+    cache = {}
     weights, x = make_inputs(w, mode)
+    cache[(w.seed, w.layers, w.bidir, w.in_dim, w.hidden, w.dtype, w.density, mode == "hlstm")] = (weights, x)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
+        # before the first CUDA call: the one-thread sample runs in a child process
+        one_thread_us = oracle_time_one_thread(args.workload)
         per_seq, reps, cores = oracle_time(w, weights, x, mode=mode)
         cpu = {"value": per_seq * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-               "sample": f"{reps} whole sequences of {w.name} (T={w.T}, one batch column each) after one warm-up"}
+               "sample": f"{reps} whole sequences of {w.name} (T={w.T}, one batch column each) after one warm-up",
+               "value_1thread": one_thread_us,
+               "sample_1thread": "3 whole sequences in a child process with OMP_NUM_THREADS=1"}
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -273,21 +485,10 @@ def run_gpu(args):
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist = dist_mod
 
-    if mode == "hlstm":
-        model = pkg.HLSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, gate_hidden=w.hidden, bidir=w.bidir,
-                          dtype=w.dtype, max_T=w.T, max_B=w.B)
-    else:
-        model = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
-                         exec_mode=mode, max_T=w.T, max_B=w.B)
     dev = torch.device("cuda", local_rank)
-    xd = torch.from_numpy(x).to(dev)
-    out = (torch.empty((w.T, w.B, w.dirs * w.hidden), device=dev),
-           torch.empty((w.layers * w.dirs, w.B, w.hidden), device=dev),
-           torch.empty((w.layers * w.dirs, w.B, w.hidden), device=dev))
     flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-
-    def step():
-        model.forward(xd, out=out)
+    case = GpuCase(torch, pkg, args.workload, dev, flush_buf, cache)
+    model = case.model
 
     def barrier():
         torch.cuda.synchronize()
@@ -296,25 +497,15 @@ def run_gpu(args):
             torch.cuda.synchronize()
 
     # ---- timed region: device-resident inputs
+    warmup = max(args.warmup, 3)
     barrier()
     with ClockSampler(local_rank) as clocks:
-        ms = time_steps(step, args.steps, max(args.warmup, 3), flush_buf, torch)
-    barrier()
-    model.check()
+        ms = case.timed(args.steps, warmup)
+        barrier()
+        # the same region once more with the library's per-kernel events (the clocks are sampled over both)
+        rec_ms, rec_n, proj_ms, stage_ms = case.kernel_split(args.steps)
     total_ms = sum(ms)
     launches_per_fwd = model.info()["launches_per_forward"]
-
-    # ---- same region again with the library's per-kernel events, for the roofline of the dominant kernel
-    model.profile_enable(True)
-    rec_ms, rec_n, proj_ms, stage_ms = 0.0, 0, 0.0, 0.0
-    for i in range(args.steps + 3):
-        flush_l2(flush_buf)
-        step()
-        n, t = model.profile_read()
-        if i >= 3:
-            rec_ms += t[pkg.LSTM_K_RECUR]; rec_n += n[pkg.LSTM_K_RECUR]
-            proj_ms += t[pkg.LSTM_K_PROJ]; stage_ms += t[pkg.LSTM_K_STAGE]
-    model.profile_enable(False)
 
     # ---- end to end through the host-buffer entry point (pinned buffers, copies inside the timing)
     xh = torch.from_numpy(x).pin_memory()
@@ -347,52 +538,81 @@ def run_gpu(args):
         ms_per_step = total_ms / args.steps
         seqs, us_per_seq, seqs_per_sec = job_throughput(world, w.B, ms_per_step)
         peak, peak_kind = measured_peaks()
-        nnz = None
-        if mode == "csr":
-            nnz = float(np.mean([sum(int(np.count_nonzero(weights[l * w.dirs + d]["mask_h"])) for d in range(w.dirs))
-                                 for l in range(w.layers)]))
-        alg_bytes = recurrence_bytes_per_launch(w, "hlstm" if mode == "hlstm" else nnz)
-        rec_avg_ms = rec_ms / max(rec_n, 1)
-        achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
-        info = model.info()
-        kernel_name, kernel_src = (("hlstm_mma_kernel", "hlstm_mma.cu") if mode == "hlstm" else
-                                   ("recur_tc_kernel", "recur_tc.cu") if info.get("recur_batched_tensor_core")
-                                   else ("recur_mma_kernel", "recur_mma.cu") if info.get("recur_register_resident")
-                                   else ("recur_kernel", "recur.cu"))
-        traffic = measured_traffic(kernel_name, args.workload, kernel_src)
+        roof = case.roofline(rec_ms, rec_n, peak, peak_kind)
+        gpu_launches = int(launches_per_fwd * args.steps)
+        if world == 1 and not args.no_legs:
+            oc = case.on_chip(min(args.steps, 20))
+            if oc is not None:
+                roof["on_chip"] = oc
         line = {
             "metric": "us_per_sequence", "value": us_per_seq, "unit": "us", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": ("bf16" if w.dtype == "bf16" else "f32"),
             "data": "synthetic",
-            "config": {"workload": w.name, "layers": w.layers, "dirs": w.dirs, "in_dim": w.in_dim, "hidden": w.hidden,
-                       "T": w.T, "B": w.B, "exec_mode": mode, "weights": w.dtype, "state": "fp32", "l2": "flushed between timed steps (256 MiB write)",
-                       "parallelism": f"replicas x{world}"},
+            "config": workload_config(w, mode, world),
             "sequences_per_sec": seqs_per_sec,
             "step_ms_p10_p50_p90": [float(np.percentile(ms, q)) for q in (10, 50, 90)],
             "clocks": clocks.summary(),
-            "gpu_launches": int(launches_per_fwd * args.steps),
+            "gpu_launches": gpu_launches,
             "e2e": {"value": e2e_ms * 1e3 / e2e_steps / seqs, "unit": "us",
                     "h2d_bytes_per_step": int(x.nbytes),
                     "d2h_bytes_per_step": int(yh.numel() * 4 + hTh.numel() * 4 + cTh.numel() * 4)},
-            "roofline": {"bound": "hbm", "kernel": f"{kernel_name} (one launch = one layer, all T steps)",
-                         "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": (achieved / peak if achieved else None), "peak_kind": f"of {peak_kind}",
-                         "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
-                         "avg_launch_ms": rec_avg_ms,
-                         "us_per_timestep": rec_avg_ms * 1e3 / w.T,
-                         "note": "the recurrent matrix stays on-chip (registers / shared memory) for the whole "
-                                 "sequence, so the fraction of the per-step HBM weight-read bound may exceed 1"},
+            "roofline": roof,
             "kernel_ms_per_forward": {"stage": stage_ms / args.steps, "projection": proj_ms / args.steps,
                                       "recurrence": rec_ms / args.steps},
             "library": model.info(),
         }
         if cpu is not None:
             line["cpu_baseline"] = cpu
+        case.close()
+        if world == 1 and not args.no_legs and args.workload == "cfg2":
+            line["legs"] = run_legs(torch, pkg, dev, flush_buf, cache, peak, peak_kind)
         print(json.dumps(line))
-    model.close()
+    else:
+        case.close()
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_legs(torch, pkg, dev, flush_buf, cache, peak, peak_kind):
+    """The other workloads of the metric, each device-timed like the headline (L2 flushed between steps, CUDA
+    events, 3 warm-up steps) with its own step count, so that the whole line stays within a minute or so."""
+    legs = {}
+    for key, name, steps in LEGS:
+        t0 = time.perf_counter()
+        try:
+            case = GpuCase(torch, pkg, name, dev, flush_buf, cache)
+        except Exception as e:      # a leg must not take the headline down with it
+            legs[key] = {"error": str(e)}
+            continue
+        try:
+            w = case.w
+            with ClockSampler(dev.index or 0) as clocks:
+                ms = case.timed(steps, 3)
+            rec_ms, rec_n, proj_ms, stage_ms = case.kernel_split(min(steps, 5))
+            nk = min(steps, 5)
+            p50 = float(np.percentile(ms, 50))
+            legs[key] = {
+                "config": workload_config(w, case.mode),
+                "steps": steps, "warmup": 3,
+                "step_ms_p10_p50_p90": [float(np.percentile(ms, q)) for q in (10, 50, 90)],
+                "ms_per_call": float(np.mean(ms)),
+                "us_per_sequence": float(np.mean(ms)) * 1e3 / w.B,
+                "sequences_per_sec": w.B / (float(np.mean(ms)) * 1e-3),
+                "sequences_per_sec_p50": w.B / (p50 * 1e-3),
+                "gpu_launches": int(case.model.info()["launches_per_forward"] * steps),
+                "kernel_ms_per_forward": {"stage": stage_ms / nk, "projection": proj_ms / nk, "recurrence": rec_ms / nk},
+                "roofline": case.roofline(rec_ms, rec_n, peak, peak_kind),
+                "clocks": clocks.summary(),
+                "wall_s": None,
+            }
+        except Exception as e:
+            legs[key] = {"error": str(e)}
+        finally:
+            case.close()
+        if isinstance(legs[key], dict) and "wall_s" in legs[key]:
+            legs[key]["wall_s"] = round(time.perf_counter() - t0, 2)
+    return legs
 
 
 def lhp_analysis(hs, lat, eps):
@@ -409,13 +629,15 @@ def run_sweep(args):
     """Latency against hidden width with the hysteresis analysis (paper, Section 3).  Shape "cfg3": one
     layer, input = hidden = H, T = 35, batch 1 (the recurrent stack of Figure 2's kind).  Shape "ds2": the
     speech-model stack (5 bidirectional layers, 1312 -> H, then 2H -> H, T = 400) at batch 16, the
-    setting of the paper's Figure 3."""
+    setting of the paper's Figure 3.  Two timings per size: `us_cold` (one call per event pair, L2 flushed before
+    it, mean without the slowest tenth, which resolves below the event clock's tick) and `us_warm` (enough calls
+    back to back inside one event pair to span at least 200 us, L2 warm: the serving-loop case)."""
     import torch
     import paper_1901_10997_b200 as pkg
     dev = torch.device("cuda", 0)
     flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-    outdir = ROOT / "gpurun_out"
-    outdir.mkdir(exist_ok=True)
+    outdir = Path(args.out)
+    outdir.mkdir(parents=True, exist_ok=True)
     ds2 = args.sweep_shape == "ds2"
     default_sizes = list(range(256, 1536 + 1, 16)) if ds2 else wl.config3_sizes()
     sizes = default_sizes if not args.sweep_sizes else [int(s) for s in args.sweep_sizes.split(",")]
@@ -429,7 +651,12 @@ def run_sweep(args):
         xd = torch.from_numpy(x).to(dev)
         out = (torch.empty((w.T, w.B, D * H), device=dev), torch.empty((w.layers * D, w.B, H), device=dev),
                torch.empty((w.layers * D, w.B, H), device=dev))
-        ms = time_steps(lambda: m.forward(xd, out=out), args.steps, max(args.warmup, 3), flush_buf, torch)
+        fn = lambda: m.forward(xd, out=out)
+        ms = time_steps(fn, args.steps, max(args.warmup, 3), flush_buf, torch)
+        m.check()
+        cold = trimmed_mean(ms)
+        calls = max(1, int(np.ceil(0.2 / max(cold, 1e-4))))
+        warm = time_back_to_back(fn, calls, 9 if not ds2 else 3, torch)
         m.check()
         err = None
         if args.sweep_parity and H in parity_sizes:
@@ -447,19 +674,21 @@ def run_sweep(args):
                 err = max(wl.rel_err(g.cpu().numpy(), r)[0] for g, r in zip(out, ref))
         info = m.info()
         m.close()
-        rows.append({"H": H, "us_p50": float(np.percentile(ms, 50)) * 1e3, "us_p10": float(np.percentile(ms, 10)) * 1e3,
+        rows.append({"H": H, "us_cold": cold * 1e3, "us_warm": warm * 1e3, "calls_per_event_pair": calls,
+                     "us_p50": float(np.percentile(ms, 50)) * 1e3, "us_p10": float(np.percentile(ms, 10)) * 1e3,
                      "us_p90": float(np.percentile(ms, 90)) * 1e3, "rows_streamed": info["rows_streamed"],
                      "threads": info["threads"], "batched_tensor_core": info.get("recur_batched_tensor_core"),
                      "max_rel_err": err})
         print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
     hs = [r["H"] for r in rows]
-    lat = [r["us_p50"] for r in rows]
     label = ("ds2 sweep: 5 bidirectional layers, 1312 -> H, T = 400, B = 16, bf16 weights; us per call (16 utterances)" if ds2
              else "cfg3 sweep: 1 layer, in = hidden = H, T = 35, B = 1, bf16 weights")
     res = {"workload": label, "steps": args.steps, "points": rows}
-    for eps in (0.0, 0.005):
-        lhps, red = lhp_analysis(hs, lat, eps)
-        res[f"lhp_eps_{eps:g}"] = {"lhps": lhps, "count": len(lhps), "redundancy_percent": red}
+    for which in ("us_warm", "us_cold"):
+        lat = [r[which] for r in rows]
+        for eps in (0.0, 0.005):
+            lhps, red = lhp_analysis(hs, lat, eps)
+            res[f"lhp_{which}_eps_{eps:g}"] = {"lhps": lhps, "count": len(lhps), "redundancy_percent": red}
     (outdir / ("sweep_ds2_b16.json" if ds2 else "sweep_cfg3.json")).write_text(json.dumps(res, indent=1))
     print(json.dumps({k: v for k, v in res.items() if k != "points"}))
 
@@ -467,14 +696,16 @@ def run_sweep(args):
 def run_matmul_sweep(args):
     """The paper's Figures 1 and 2 on this GPU: one square matrix W [d x d] times a batch of 16 dense columns,
     dense (tensor-core projection, bf16 weights) against sparse (CSR projection over the surviving weights)
-    at 90 % and 95 % sparsity, d = 128 .. 2048.  Timed with the library's per-kernel events (staging +
-    projection kernels), L2 flushed between calls."""
+    at 90 % and 95 % sparsity, d = 128 .. 2048.  Every variant is timed the same way: the whole
+    lstm_input_projection call (staging where the variant has it, product, re-layout of the result), enough
+    calls back to back inside one event pair to span 200 us (`_us`, L2 warm) and, beside it, one call per event
+    pair with L2 flushed (`_cold_us`, mean without the slowest tenth)."""
     import torch
     import paper_1901_10997_b200 as pkg
     dev = torch.device("cuda", 0)
     flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-    outdir = ROOT / "gpurun_out"
-    outdir.mkdir(exist_ok=True)
+    outdir = Path(args.out)
+    outdir.mkdir(parents=True, exist_ok=True)
     rows = []
     for dsz in range(128, 2048 + 1, 64):
         H = dsz // 4
@@ -486,26 +717,64 @@ def run_matmul_sweep(args):
             m = pkg.LSTM(weights, layers=1, in_dim=dsz, hidden=H, dtype="bf16", exec_mode=mode, max_T=16, max_B=1)
             xd = torch.from_numpy(x).to(dev)
             out = torch.empty((16, 1, 1, 4 * H), device=dev)
-            m.profile_enable(True)
-            ts = []
-            for i in range(args.steps + max(args.warmup, 3)):
-                flush_l2(flush_buf)
-                m.input_projection(xd, out=out)
-                _n, t = m.profile_read()
-                if i >= max(args.warmup, 3):
-                    ts.append((t[pkg.LSTM_K_STAGE] + t[pkg.LSTM_K_PROJ]) * 1e3)
+            fn = lambda: m.input_projection(xd, out=out)
+            ms = time_steps(fn, args.steps, max(args.warmup, 3), flush_buf, torch)
+            cold = trimmed_mean(ms)
+            calls = max(1, int(np.ceil(0.2 / max(cold, 1e-4))))
+            warm = time_back_to_back(fn, calls, 9, torch)
             m.check()
             if args.sweep_parity:
                 import oracle
                 ref = oracle.input_projection(weights, x, bidir=False, hidden=H)
                 row[label + "_err"] = wl.rel_err(out.cpu().numpy().reshape(ref.shape), ref)[1]
             m.close()
-            row[label + "_us"] = float(np.percentile(ts, 50))
+            row[label + "_us"] = warm * 1e3
+            row[label + "_cold_us"] = cold * 1e3
         rows.append(row)
         print(json.dumps(row), file=sys.stderr, flush=True)
     (outdir / "matmul_sweep.json").write_text(json.dumps({"batch": 16, "steps": args.steps, "points": rows}, indent=1))
-    wins = sum(1 for r in rows if r["csr_05_us"] < r["dense_tc_us"])
-    print(json.dumps({"points": len(rows), "sparse_95_faster_than_dense_at": wins}))
+    summary = {"points": len(rows)}
+    for which in ("_us", "_cold_us"):
+        summary["sparse_95_faster_than_dense" + which] = sum(1 for r in rows if r["csr_05" + which] < r["dense_tc" + which])
+        summary["sparse_90_faster_than_dense" + which] = sum(1 for r in rows if r["csr_10" + which] < r["dense_tc" + which])
+    print(json.dumps(summary))
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def spawn_replicas(args):
+    """`--gpus N` without a launcher: start the N ranks (one process per GPU) under torch's own launcher on
+    127.0.0.1 and hand back its exit code; rank 0 prints the job's single JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), str(Path(__file__).resolve()), *sys.argv[1:]]
+    return subprocess.call(cmd)
+
+
+def run_replica_check(args):
+    """The rank bookkeeping of the N-replica run with no GPU work (gloo): every rank joins the group, takes part
+    in the barrier and the max-over-ranks reduction of a made-up step time (10 + rank ms), rank 0 prints."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    d = None
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+        d = dist
+    total_ms, = max_over_ranks([10.0 + rank], d, torch.device("cpu"))
+    seqs, us_per_seq, per_sec = job_throughput(world, 1, total_ms)
+    if rank == 0:
+        print(json.dumps({"replica_check": True, "n_gpus": world, "ms_per_step": total_ms, "sequences_per_step": seqs,
+                          "value": us_per_seq, "sequences_per_sec": per_sec}))
+    if d is not None:
+        dist.destroy_process_group()
 
 
 def main():
@@ -516,13 +785,20 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-legs", action="store_true")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--matmul-sweep", action="store_true")
     ap.add_argument("--sweep-sizes", default="")
     ap.add_argument("--sweep-shape", default="cfg3", choices=["cfg3", "ds2"])
     ap.add_argument("--sweep-parity", action="store_true")
+    ap.add_argument("--out", default=str(ROOT / "bench_out"))
+    ap.add_argument("--replica-check", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.sweep or args.matmul_sweep):
+        raise SystemExit(spawn_replicas(args))
+    if args.replica_check:
+        run_replica_check(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.sweep:
         run_sweep(args)

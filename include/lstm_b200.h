@@ -197,6 +197,20 @@ LSTM_API int lstm_profile_enable(lstm_handle *h, int on);
 LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
 
 /*
+ * Step-cost probe of the register-resident recurrent kernel (bf16 dense LSTM handles, calls with one sequence;
+ * calls with more run normally).  A recurrent step is a chain: wait for the other CTAs' h words -> tensor-core products ->
+ * CTA barrier, reduction, gate functions -> publish.  With a non-zero mask the following lstm_forward calls
+ * leave parts of that chain out, so that timing them shows what each part costs (the "empty step": exchange
+ * only, is the floor no kernel of this structure can go below).  Bits: LSTM_PROBE_NO_PRODUCTS (no tensor
+ * instructions), LSTM_PROBE_NO_GATES (no reduction, gate functions or output stores; every unit still
+ * publishes a word per step), LSTM_PROBE_NO_EXCHANGE (no waiting for other CTAs).  OUTPUTS ARE UNDEFINED
+ * while a mask is set; 0 restores normal operation.  LSTM_ERR_UNSUPPORTED for handles that run another
+ * recurrent kernel.  Every wait stays bounded in every mode.
+ */
+enum { LSTM_PROBE_NO_PRODUCTS = 1, LSTM_PROBE_NO_GATES = 2, LSTM_PROBE_NO_EXCHANGE = 4 };
+LSTM_API int lstm_probe(lstm_handle *h, int parts_left_out);
+
+/*
  * Read-only facts about how the handle runs (for reports): writes up to n values into out and
  * returns the number available.  Order: [0] SM count, [1] CTAs of the recurrent kernel per direction,
  * [2] threads per CTA, [3] dynamic shared memory bytes per CTA at max_B, [4] recurrent-matrix rows

@@ -15,6 +15,7 @@ LSTM_F32, LSTM_BF16W_F32S = 0, 1
 LSTM_DENSE, LSTM_CSR = 0, 1
 LSTM_OK, LSTM_ERR_INVALID, LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT = range(6)
 LSTM_K_STAGE, LSTM_K_PROJ, LSTM_K_RECUR, LSTM_K_COUNT = 0, 1, 2, 3
+LSTM_PROBE_NO_PRODUCTS, LSTM_PROBE_NO_GATES, LSTM_PROBE_NO_EXCHANGE = 1, 2, 4
 
 _LIB_PATH = Path(__file__).resolve().parent / "liblstm_b200.so"
 _lib = None
@@ -74,6 +75,8 @@ def load_library():
         lib.lstm_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), ci]
         lib.lstm_selftest_timeout.restype = ci
         lib.lstm_selftest_timeout.argtypes = [vp, ci, ctypes.c_longlong]
+        lib.lstm_probe.restype = ci
+        lib.lstm_probe.argtypes = [vp, ci]
         lib.lstm_forward_noalloc.restype = ci
         lib.lstm_forward_noalloc.argtypes = [vp, vp, vp, ci, ci, vp, ci, ci, vp, vp, vp, vp, vp, vp, ctypes.c_char_p, ci]
         pi, pd, pf = ctypes.POINTER(ci), ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_float)
@@ -133,6 +136,10 @@ def lstm_destroy(handle):
 
 def lstm_selftest_timeout(handle, cta, spin_limit=0):
     return load_library().lstm_selftest_timeout(handle, cta, spin_limit)
+
+
+def lstm_probe(handle, parts_left_out):
+    return load_library().lstm_probe(handle, int(parts_left_out))
 
 
 def lstm_profile_enable(handle, on):
@@ -336,6 +343,10 @@ class LSTM:
 
     def selftest_timeout(self, cta, spin_limit=0):
         self._check(lstm_selftest_timeout(self._handle, cta, spin_limit))
+
+    def probe(self, parts_left_out=0):
+        """Step-cost measurement: leave parts of the recurrent step out (outputs undefined until reset to 0)."""
+        self._check(lstm_probe(self._handle, parts_left_out))
 
     def profile_enable(self, on=True):
         self._check(lstm_profile_enable(self._handle, on))

@@ -73,6 +73,7 @@ struct lstm_handle {
     long long spin_limit = 2000000000LL;
     long long spin_limit_default = 2000000000LL;
     int withhold_cta = -1;             // failure-path self-test (lstm_selftest_timeout)
+    int probe = 0;                     // step-cost measurement (lstm_probe): parts of the recurrent step left out
     cudaStream_t last_stream = nullptr;
     // host-buffer variant staging
     float *hx = nullptr, *hy = nullptr, *hh0 = nullptr, *hc0 = nullptr, *hhT = nullptr, *hcT = nullptr;
@@ -1025,6 +1026,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             h->stamp_next += (unsigned)T + 1u;
             m.spin_limit = h->spin_limit;
             m.withhold_cta = h->withhold_cta;
+            m.probe = B == 1 ? h->probe : 0;
             for (int d = 0; d < D; ++d) m.wfrag[d] = ly.wfrag[d];
             m.G = h->G;
             m.g_split_stride = (long long)M * N;
@@ -1163,6 +1165,16 @@ int lstm_selftest_timeout(lstm_handle *h, int cta, long long spin_limit)
     if (cta >= h->ncta_dir * h->D) return fail(h, LSTM_ERR_INVALID, "cta %d outside the launch of %d CTAs", cta, h->ncta_dir * h->D);
     h->withhold_cta = cta < 0 ? -1 : cta;
     h->spin_limit = spin_limit > 0 ? spin_limit : h->spin_limit_default;
+    return LSTM_OK;
+}
+
+int lstm_probe(lstm_handle *h, int parts_left_out)
+{
+    if (!h) return LSTM_ERR_INVALID;
+    if (parts_left_out < 0 || parts_left_out > 7) return fail(h, LSTM_ERR_INVALID, "probe mask %d outside 0..7", parts_left_out);
+    if (parts_left_out && (!h->use_mma || h->Hh))
+        return fail(h, LSTM_ERR_UNSUPPORTED, "only the register-resident recurrent kernel of an LSTM handle has probe modes");
+    h->probe = parts_left_out;
     return LSTM_OK;
 }
 

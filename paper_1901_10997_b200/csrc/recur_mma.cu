@@ -110,9 +110,12 @@ constexpr int kChunk = 4;     // batch rows per pass: hi and lo parts fill the 8
 // out of the single-row instantiation, whose registers are all spoken for.
 // ONE: a single sequence (B = 1): the batch-row arithmetic folds away at compile time.
 // POLL3: a lane polls three words per round instead of four (single sequence, at most 96 columns per warp).
-template <int MT, int NKR, int NW, bool STAGED, bool ONE, bool POLL3>
+// PROBE: the measurement build of the single-sequence variants, which honours a.probe (parts of a step left
+// out); in every other instantiation the probe tests fold away, so the production step carries none of them.
+template <int MT, int NKR, int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE = false>
 __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArgs a)
 {
+    const int probe = PROBE ? a.probe : 0;
     constexpr int NT = NW * 32;
     constexpr int RP = MT * 16 + 8;          // row pitch of the partial sums: conflict-free writes
     constexpr int WS = 4 * RP + 4;           // pitch between warps: the readers of one row spread over the banks
@@ -232,7 +235,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                         Bw[dof + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
                     }
                 }
-            } else if (a.probe & kProbeNoExchange) {
+            } else if (probe & kProbeNoExchange) {
                 // measurement only: no wait for the other CTAs, the operand keeps whatever it holds
             } else if (STAGED) {
                 // Several batch rows: too many words per lane to hold in registers at once, and polling
@@ -340,7 +343,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
             for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
-            if (!(a.probe & kProbeNoProducts)) {
+            if (!(probe & kProbeNoProducts)) {
 #pragma unroll
                 for (int i = 0; i < NKR; ++i) {
                     const unsigned bv0 = Bw32[i * 64 + g * 8 + tig];
@@ -366,7 +369,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
             // ---- all partial sums of this pass are in place (two barriers and two buffers alternate)
             bar_sync(1 + (it & 1), nbar);
 
-            if (fin_warp && (a.probe & kProbeNoGates)) {
+            if (fin_warp && (probe & kProbeNoGates)) {
                 // measurement only: the exchange without the reduction, the gate functions and the outputs
                 if (fq == 0 && fpart == 0 && fb < nb && (int)blockIdx.x != a.withhold_cta)
                     st_relaxed_u64(xch_d + ((size_t)(s & 1) * B + b0 + fb) * H + u0 + warp,
@@ -419,33 +422,36 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 
 typedef void (*KernelFn)(const RecurMmaArgs);
 
-template <int MT, int NW, bool STAGED, bool ONE, bool POLL3>
+template <int MT, int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE>
 KernelFn pick_nkr(int nkr)
 {
     switch (nkr) {
-        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE, POLL3>;
-        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE, POLL3>;
-        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE, POLL3>;
-        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE, (POLL3 && false)>;     // 128 columns per warp: four words
+        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE, POLL3, PROBE>;
+        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE, POLL3, PROBE>;
+        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE, POLL3, PROBE>;
+        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE, (POLL3 && false), PROBE>;     // 128 columns per warp: four words
         default: return nullptr;
     }
 }
-template <int NW, bool STAGED, bool ONE, bool POLL3>
+template <int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE = false>
 KernelFn pick_mt(int mt, int nkr)
 {
     switch (mt) {
-        case 1: return pick_nkr<1, NW, STAGED, ONE, POLL3>(nkr);
-        case 2: return pick_nkr<2, NW, STAGED, ONE, POLL3>(nkr);
-        case 3: return pick_nkr<3, NW, STAGED, ONE, POLL3>(nkr);
-        case 4: return pick_nkr<4, NW, STAGED, ONE, POLL3>(nkr);
+        case 1: return pick_nkr<1, NW, STAGED, ONE, POLL3, PROBE>(nkr);
+        case 2: return pick_nkr<2, NW, STAGED, ONE, POLL3, PROBE>(nkr);
+        case 3: return pick_nkr<3, NW, STAGED, ONE, POLL3, PROBE>(nkr);
+        case 4: return pick_nkr<4, NW, STAGED, ONE, POLL3, PROBE>(nkr);
         default: return nullptr;
     }
 }
 // variant 0: several rows polled from registers, 1: several rows staged in shared memory, 2: one sequence,
-// 3: one sequence with at most 96 columns per warp (three polled words per lane)
+// 3: one sequence with at most 96 columns per warp (three polled words per lane); 4, 5: the measurement
+// builds of 2 and 3
 KernelFn pick(int mt, int nkr, int nw, int variant)
 {
     if (!recur_mma_shape_ok(mt, nkr, nw)) return nullptr;
+    if (variant == 4) return nw == 8 ? pick_mt<8, false, true, false, true>(mt, nkr) : pick_mt<16, false, true, false, true>(mt, nkr);
+    if (variant == 5) return nw == 8 ? pick_mt<8, false, true, true, true>(mt, nkr) : pick_mt<16, false, true, true, true>(mt, nkr);
     if (variant == 1) return nw == 8 ? pick_mt<8, true, false, false>(mt, nkr) : pick_mt<16, true, false, false>(mt, nkr);
     if (variant == 2) return nw == 8 ? pick_mt<8, false, true, false>(mt, nkr) : pick_mt<16, false, true, false>(mt, nkr);
     if (variant == 3) return nw == 8 ? pick_mt<8, false, true, true>(mt, nkr) : pick_mt<16, false, true, true>(mt, nkr);
@@ -471,7 +477,7 @@ size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int 
 
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 {
-    for (int variant = 0; variant < 4; ++variant) {
+    for (int variant = 0; variant < 6; ++variant) {
         KernelFn fn = pick(mt, nkr, nw, variant);
         if (!fn) return cudaErrorInvalidValue;
         const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
@@ -482,7 +488,11 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st)
 {
-    const int variant = a.staged ? 1 : a.B != 1 ? 0 : (nkr + a.nkw_smem) * 16 <= 96 ? 3 : 2;
+    int variant = a.staged ? 1 : a.B != 1 ? 0 : (nkr + a.nkw_smem) * 16 <= 96 ? 3 : 2;
+    if (a.probe) {
+        if (variant < 2) return cudaErrorInvalidValue;      // probe modes exist for the single-sequence variants only
+        variant += 2;
+    }
     KernelFn fn = pick(mt, nkr, nw, variant);
     if (!fn) return cudaErrorInvalidValue;
     RecurMmaArgs copy = a;

@@ -68,3 +68,18 @@ def test_reference_arm_runs_on_rank0_only(monkeypatch, capsys):
     monkeypatch.setenv("RANK", "1")
     bench.run_reference(A)
     assert capsys.readouterr().out == ""
+
+
+def test_gpus_flag_alone_starts_the_ranks():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks itself; the bookkeeping-only mode
+    (gloo, no GPU work) shows that both joined: n_gpus = 2 and the step time is the slower rank's."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--replica-check"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["ms_per_step"] == 11.0 and d["sequences_per_step"] == 2
