@@ -333,7 +333,7 @@ def kernel_of(info, mode):
     if mode == "hlstm":
         return "hlstm_mma_kernel", "hlstm_mma.cu"
     if mode == "csr":
-        return ("recur_csr_kernel", "recur_csr.cu") if info.get("recur_register_resident") else ("recur_kernel", "recur.cu")
+        return ("recur_csr_kernel", "recur_csr.cu") if info.get("recur_csr_register_resident") else ("recur_kernel", "recur.cu")
     if info.get("recur_batched_tensor_core"):
         return "recur_tc_kernel", "recur_tc.cu"
     if info.get("recur_register_resident"):

@@ -99,7 +99,7 @@ typedef struct {
  *   cuda_stream: a cudaStream_t (NULL = default stream) used for the uploads.
  * Synchronises the stream before returning.  On failure *out is NULL.
  * Environment switches read at create time (for measurements and tests; unset = the library chooses):
- *   LSTM_B200_RECUR = simt  shared-memory recurrent kernel instead of the register-resident one (bf16 dense)
+ *   LSTM_B200_RECUR = simt  shared-memory recurrent kernel instead of the register-resident one (bf16 dense or CSR)
  *                   = mma   no batched tensor-core recurrence (batches above four run as passes of four)
  *                   = tc1   batched tensor-core recurrence without cluster pairs
  *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
@@ -221,7 +221,10 @@ LSTM_API int lstm_probe(lstm_handle *h, int parts_left_out);
  * [10] 16-column weight tiles per warp held in registers, [11] per warp held in shared memory,
  * [12] 1 if a call at max_B runs the batched tensor-core (tcgen05) recurrence: bf16 dense LSTM handles use
  * it for batches of 5 to 64 sequences where its operand ring fits beside the resident slice, and the
- * register-resident kernel (passes of four sequences) otherwise.
+ * register-resident kernel (passes of four sequences) otherwise,
+ * [13] 1 if a CSR handle runs the register-resident sparse kernel (bf16 storage, at most 16 units per CTA,
+ * lane lists short enough for registers), 0 for the shared-memory CSR kernel, [14] its entry slots per lane,
+ * [15] shared-memory wavefronts per step and CTA that its gathers lose to bank conflicts (worst CTA).
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 
@@ -254,6 +257,25 @@ LSTM_API int lstm_nearest_lhp(const int *sizes, const double *latency, int n, do
  */
 LSTM_API int lstm_fold_input_affine(const float *wx, const float *b, int rows, int cols, const float *scale,
                                     const float *shift, float *wx_out, float *b_out);
+
+/*
+ * Create-time layout of one pruned recurrent matrix for the register-resident sparse kernel (Section 4: the
+ * mask-based scheme leaves an unstructured pattern of surviving weights), as a host-only call so that the
+ * layout can be inspected and tested without a GPU; lstm_create runs the same code.
+ *   rowptr/col/val: CSR of Wh [4*hidden x hidden], rows in gate-block order q*hidden + j, columns increasing.
+ *   The hidden units are split evenly over `ctas` CTAs of `warps` (8 or 16) warps; warp w owns the columns
+ *   [w*kspan, (w+1)*kspan) (kspan a multiple of 32 with warps*kspan >= hidden); inside a warp every lane owns
+ *   at most two of the CTA's 4*units rows, longest rows dealt first.
+ * Outputs (each may be NULL): *longest = entries of the longest lane list; rows[ctas*warps*32] = the lanes' two
+ * local rows (4*unit + gate in byte 0 and byte 1, 0xff = none); entries[ctas*warps*slots*32] = the lists padded to
+ * `slots` (>= *longest) words {bf16 value:16 | second-row flag:1 | 4*(column - w*kspan):15}, stored
+ * [cta][warp][slot][lane], ordered so that the 32 gathers of a slot fall into different shared-memory banks
+ * where the pattern allows; *conflict_wavefronts = extra wavefronts per step that remain (worst CTA).
+ * LSTM_ERR_UNSUPPORTED when a CTA would own more than `warps` units; LSTM_ERR_INVALID for bad arguments.
+ */
+LSTM_API int lstm_csr_lane_layout(const int32_t *rowptr, const int32_t *col, const float *val, int hidden, int ctas,
+                                  int warps, int kspan, int slots, uint32_t *entries, uint32_t *rows, int *longest,
+                                  long long *conflict_wavefronts);
 
 /*
  * Forward pass without any allocation (the paper has no counterpart: this exists for deployment).

@@ -86,6 +86,8 @@ def load_library():
         lib.lstm_nearest_lhp.argtypes = [pi, pd, ci, ctypes.c_double, ci, pi]
         lib.lstm_fold_input_affine.restype = ci
         lib.lstm_fold_input_affine.argtypes = [pf, pf, ci, ci, pf, pf, pf, pf]
+        lib.lstm_csr_lane_layout.restype = ci
+        lib.lstm_csr_lane_layout.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, pi, ctypes.POINTER(ctypes.c_longlong)]
         _lib = lib
     return _lib
 
@@ -154,11 +156,12 @@ def lstm_profile_read(handle):
 
 
 def lstm_info(handle):
-    out = (ctypes.c_int64 * 16)()
-    n = load_library().lstm_info(handle, out, 16)
+    out = (ctypes.c_int64 * 32)()
+    n = load_library().lstm_info(handle, out, 32)
     keys = ["sm_count", "ctas_per_dir", "threads", "smem_bytes", "rows_resident", "rows_streamed",
             "proj_splits", "proj_tensor_core", "launches_per_forward", "recur_register_resident",
-            "col_tiles_in_registers", "col_tiles_in_smem", "recur_batched_tensor_core"]
+            "col_tiles_in_registers", "col_tiles_in_smem", "recur_batched_tensor_core",
+            "recur_csr_register_resident", "csr_slots_per_lane", "csr_bank_conflict_wavefronts"]
     return {k: int(out[i]) for i, k in enumerate(keys[:n])}
 
 
@@ -198,6 +201,22 @@ def lstm_fold_input_affine(wx, b, scale, shift):
     ptr = lambda a: None if a is None else a.ctypes.data_as(pf)
     rc = load_library().lstm_fold_input_affine(ptr(wx), ptr(b), rows, cols, ptr(scale), ptr(shift), ptr(wx_out), ptr(b_out))
     return rc, wx_out, b_out
+
+
+def lstm_csr_lane_layout(rowptr, col, val, hidden, ctas, warps, kspan, slots=None):
+    """Returns (code, longest, rows, entries, conflict_wavefronts); with ``slots`` None only the list lengths and
+    rows are computed (entries is None).  rows: uint32 [ctas, warps, 32]; entries: uint32 [ctas, warps, slots, 32]."""
+    rowptr = np.ascontiguousarray(rowptr, np.int32)
+    col = np.ascontiguousarray(col, np.int32)
+    val = np.ascontiguousarray(val, np.float32)
+    rows = np.zeros((ctas, warps, 32), np.uint32)
+    longest = ctypes.c_int(0)
+    conflicts = ctypes.c_longlong(0)
+    entries = None if slots is None else np.zeros((ctas, warps, slots, 32), np.uint32)
+    rc = load_library().lstm_csr_lane_layout(rowptr.ctypes.data, col.ctypes.data, val.ctypes.data, hidden, ctas, warps, kspan,
+                                             0 if slots is None else slots, None if entries is None else entries.ctypes.data,
+                                             rows.ctypes.data, ctypes.byref(longest), ctypes.byref(conflicts))
+    return rc, int(longest.value), rows, entries, int(conflicts.value)
 
 
 def lstm_forward_noalloc(wx, wh, b, in_dim, hidden, x, T, B, h0, c0, y, hT, cT, stream=0):

@@ -2,6 +2,8 @@
 // variant, status and measurement support.  See include/lstm_b200.h for the contract.
 #include "../../include/lstm_b200.h"
 #include "common.cuh"
+#include "csr_pack.h"
+#include "device_util.cuh"
 
 #include <algorithm>
 #include <cmath>
@@ -35,6 +37,9 @@ struct Layer {
     uint4 *frag2[2] = {nullptr, nullptr};  // H-LSTM: fragments of the gate output matrices W
     float *bias_out = nullptr;             // H-LSTM: [D][H][4] bias of the gate pre-activations
     int csr_max_slice_entries = 0;     // largest per-CTA slice (entries, padded)
+    unsigned *csr_reg_ent[2] = {nullptr, nullptr};   // register-resident sparse kernel: [cta][warp][slots][32] entry words
+    unsigned *csr_reg_rows[2] = {nullptr, nullptr};  //   and the lanes' rows [cta][warp][32]
+    CsrLaneLists csr_lists[2];         // host side, until the slot count of the handle is known
     ProjTcPlan plan;                   // tensor-core projection plan for plan_M rows
     int plan_M = -1;
 };
@@ -50,6 +55,10 @@ struct lstm_handle {
     // register-resident recurrent kernel (bf16 dense): row tiles, column tiles per warp in registers and
     // in shared memory, warps per CTA
     bool use_mma = false;
+    // register-resident sparse kernel (bf16, CSR execution): warps, columns per warp, row tiles, entry slots per lane
+    bool use_csr_reg = false;
+    int csr_nw = 0, csr_kspan = 0, csr_mt = 0, csr_slots = 0;
+    long long csr_conflicts = 0;       // shared-memory wavefronts per step and CTA lost to bank conflicts (worst CTA, worst matrix)
     int mma_mt = 0, mma_nkr = 0, mma_nks = 0, mma_nw = 0;
     // batched tensor-core recurrence (more than four batch rows): weight-tile rows, K blocks, planes, stamps
     bool seq_dirs = false;             // bidirectional layers run one direction after the other, each on all SMs
@@ -108,22 +117,6 @@ int check_device(lstm_handle *h)
     if (dev != h->device)
         return fail(h, LSTM_ERR_INVALID, "the handle belongs to device %d but device %d is current; nothing launched", h->device, dev);
     return LSTM_OK;
-}
-
-inline uint16_t f32_to_bf16_rne(float f)
-{
-    uint32_t u;
-    memcpy(&u, &f, 4);
-    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);   // NaN stays NaN
-    u += 0x7fffu + ((u >> 16) & 1u);
-    return (uint16_t)(u >> 16);
-}
-inline float bf16_to_f32(uint16_t b)
-{
-    uint32_t u = (uint32_t)b << 16;
-    float f;
-    memcpy(&f, &u, 4);
-    return f;
 }
 
 // Returns a host-readable view of n bytes at p (copying from the device when p is device memory).
@@ -341,7 +334,7 @@ void plan_mma(lstm_handle *h)
 
 int max_b_fits(const lstm_handle *h)
 {
-    if (h->use_mma) return 1;
+    if (h->use_mma || h->use_csr_reg) return 1;
     // the staging buffers and the c state must fit even when no weight is resident
     const size_t budget = (size_t)h->smem_optin - 64;
     const size_t c_bytes = (size_t)round_up(h->upc * h->max_B, 4) * 4;
@@ -349,11 +342,40 @@ int max_b_fits(const lstm_handle *h)
     return (size_t)2 * h->Hs * 4 + c_bytes + rp <= budget;
 }
 
+// Operand-A fragments of a [4U x K] matrix whose row q*U + u is gate q of unit u: per CTA (units split
+// evenly over ncta CTAs) [warp][column tile][row tile][lane] x 4 words, local row = 4 * unit + gate,
+// zero beyond the CTA's units and beyond column K.
+std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int NW, int nkw, int MT)
+{
+    std::vector<uint32_t> f((size_t)ncta * NW * nkw * MT * 32 * 4, 0u);
+    size_t o = 0;
+    for (int c = 0; c < ncta; ++c) {
+        int u0, nu; unit_range_host(U, ncta, c, u0, nu);
+        auto wv = [&](int r, int k) -> uint32_t {
+            if (r >= 4 * nu || k >= K) return 0u;
+            return f32_to_bf16_rne(m[(size_t)((r & 3) * U + u0 + (r >> 2)) * K + k]);
+        };
+        for (int wp = 0; wp < NW; ++wp)
+            for (int i = 0; i < nkw; ++i)
+                for (int mt = 0; mt < MT; ++mt)
+                    for (int lane = 0; lane < 32; ++lane) {
+                        const int g = lane >> 2, p2 = (lane & 3) * 2;
+                        const int r0 = mt * 16 + g, r1 = r0 + 8;
+                        const int ka = (wp * nkw + i) * 16 + p2, kb = ka + 8;
+                        f[o++] = wv(r0, ka) | (wv(r0, ka + 1) << 16);
+                        f[o++] = wv(r1, ka) | (wv(r1, ka + 1) << 16);
+                        f[o++] = wv(r0, kb) | (wv(r0, kb + 1) << 16);
+                        f[o++] = wv(r1, kb) | (wv(r1, kb + 1) << 16);
+                    }
+    }
+    return f;
+}
+
 void free_all(lstm_handle *h)
 {
     for (auto &ly : h->layers) {
         cudaFree(ly.wx); cudaFree(ly.bias); cudaFree(ly.wx_rowptr); cudaFree(ly.wx_ent);
-        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); cudaFree(ly.frag2[d]); }
+        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); cudaFree(ly.frag2[d]); cudaFree(ly.csr_reg_ent[d]); cudaFree(ly.csr_reg_rows[d]); }
         cudaFree(ly.bias_out); cudaFree(ly.wtc);
     }
     cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
@@ -420,6 +442,17 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
     plan_mma(h);
+    if (csr && bf16) {
+        // the register-resident sparse kernel: at most 16 units per CTA (warp w finishes unit w, a lane owns at
+        // most two of the 4 * units rows); the entry slots per lane are known once every matrix has been laid out
+        const char *env = getenv("LSTM_B200_RECUR");
+        const int nw = (h->upc <= 8 && H <= 512) ? 8 : 16;
+        const int kspan = round_up((H + nw - 1) / nw, 32), mt = (4 * h->upc + 15) / 16;
+        if (!(env && strcmp(env, "simt") == 0) && h->upc <= nw &&
+            recur_csr_reg_smem_bytes(nw, kspan, mt, h->upc, max_B) <= (size_t)h->smem_optin - 64) {
+            h->use_csr_reg = true; h->csr_nw = nw; h->csr_kspan = kspan; h->csr_mt = mt;
+        }
+    }
     // does the batched tensor-core recurrence fit with the current split of the SMs?
     auto tcb_fits = [&](int *kbs, int *stages) -> bool {
         const char *env = getenv("LSTM_B200_RECUR");
@@ -504,30 +537,7 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                 if (rc) break;
                 const size_t n = (size_t)H * 4 * h->Hp8;
                 if (h->use_mma) {
-                    // operand-A fragments: [cta][warp][column tile][row tile][lane] x 4 words; local row
-                    // r = 4 * unit + gate, zero beyond the CTA's units and beyond column H
-                    const int NW = h->mma_nw, nkw = h->mma_nkr + h->mma_nks, MT = h->mma_mt;
-                    std::vector<uint32_t> f((size_t)h->ncta_dir * NW * nkw * MT * 32 * 4, 0u);
-                    size_t o = 0;
-                    for (int c = 0; c < h->ncta_dir; ++c) {
-                        int u0, nu; unit_range_host(H, h->ncta_dir, c, u0, nu);
-                        auto wv = [&](int r, int k) -> uint32_t {
-                            if (r >= 4 * nu || k >= H) return 0u;
-                            return f32_to_bf16_rne(m[(size_t)((r & 3) * H + u0 + (r >> 2)) * H + k]);
-                        };
-                        for (int wp = 0; wp < NW; ++wp)
-                            for (int i = 0; i < nkw; ++i)
-                                for (int mt = 0; mt < MT; ++mt)
-                                    for (int lane = 0; lane < 32; ++lane) {
-                                        const int g = lane >> 2, p2 = (lane & 3) * 2;
-                                        const int r0 = mt * 16 + g, r1 = r0 + 8;
-                                        const int ka = (wp * nkw + i) * 16 + p2, kb = ka + 8;
-                                        f[o++] = wv(r0, ka) | (wv(r0, ka + 1) << 16);
-                                        f[o++] = wv(r1, ka) | (wv(r1, ka + 1) << 16);
-                                        f[o++] = wv(r0, kb) | (wv(r0, kb + 1) << 16);
-                                        f[o++] = wv(r1, kb) | (wv(r1, kb + 1) << 16);
-                                    }
-                    }
+                    const std::vector<uint32_t> f = pack_fragments(m.data(), H, H, h->ncta_dir, h->mma_nw, h->mma_nkr + h->mma_nks, h->mma_mt);
                     rc = upload(h, (uint32_t **)&ly.wfrag[d], f.data(), f.size() * 4, st, "recurrent weight fragments");
                     if (rc == LSTM_OK) cudaStreamSynchronize(st);
                 } else if (bf16) {
@@ -580,6 +590,10 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
                 snprintf(name, sizeof name, "wh[layer %d, dir %d]", l, d);
                 rc = matrix_to_csr(h, 4 * H, H, src.wh, src.mask_h, src.wh_rowptr, src.wh_col, src.wh_val, ch, name);
                 if (rc) break;
+                if (h->use_csr_reg) {
+                    csr_lane_lists(ch.rowptr.data(), ch.col.data(), ch.val.data(), H, h->ncta_dir, h->csr_nw, h->csr_kspan, ly.csr_lists[d]);
+                    h->csr_slots = std::max(h->csr_slots, ly.csr_lists[d].longest);
+                }
                 std::vector<int> ptr(4 * H + 1, 0);
                 std::vector<unsigned> e16; std::vector<CsrEntry> e32;
                 for (int j = 0; j < H; ++j)
@@ -624,6 +638,29 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     }
     if (rc) return bail(rc);
 
+    if (h->use_csr_reg) {
+        // one slot count for the whole handle: the longest lane list of any matrix, rounded up to a built size
+        const int slots = recur_csr_reg_slots(std::max(h->csr_slots, 1), h->csr_nw);
+        if (slots == 0) h->use_csr_reg = false;            // lists too long for registers: the shared-memory kernel runs
+        h->csr_slots = slots;
+        for (int l = 0; l < layers && rc == LSTM_OK; ++l)
+            for (int d = 0; d < D && rc == LSTM_OK; ++d) {
+                Layer &ly = h->layers[l];
+                if (h->use_csr_reg) {
+                    long long conflicts = 0;
+                    const std::vector<unsigned> packed = csr_pack_slots(ly.csr_lists[d], h->ncta_dir, h->csr_nw, slots, h->csr_kspan, &conflicts);
+                    h->csr_conflicts = std::max(h->csr_conflicts, conflicts);
+                    rc = upload(h, &ly.csr_reg_ent[d], packed.data(), packed.size() * 4, st, "sparse recurrent entries");
+                    if (rc == LSTM_OK) rc = upload(h, &ly.csr_reg_rows[d], ly.csr_lists[d].rows.data(), ly.csr_lists[d].rows.size() * 4, st, "sparse recurrent rows");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                    cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]);       // the shared-memory kernel's copy is not needed
+                    ly.wh_ptr[d] = nullptr; ly.wh_ent[d] = nullptr;
+                }
+                ly.csr_lists[d] = CsrLaneLists();
+            }
+        if (rc) return bail(rc);
+    }
+
     // workspace
     const size_t Mmax = (size_t)max_T * max_B;
     const size_t N = (size_t)D * 4 * H;
@@ -647,7 +684,8 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     }
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
     if (rc == LSTM_OK) {
-        cudaError_t e = csr ? recur_csr_prepare(h->smem_optin - 64)
+        cudaError_t e = h->use_csr_reg ? recur_csr_reg_prepare(h->csr_slots, h->csr_nw, h->smem_optin - 64)
+                            : csr ? recur_csr_prepare(h->smem_optin - 64)
                             : h->use_mma ? recur_mma_prepare(h->mma_mt, h->mma_nkr, h->mma_nw, h->smem_optin - 64)
                                          : recur_dense_prepare(h->smem_optin - 64);
         if (e == cudaSuccess && h->use_tc) e = proj_tc_prepare();
@@ -660,35 +698,6 @@ int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir
     if (rc) return bail(rc);
     *out = h;
     return LSTM_OK;
-}
-
-// Operand-A fragments of a [4U x K] matrix whose row q*U + u is gate q of unit u: per CTA (units split
-// evenly over ncta CTAs) [warp][column tile][row tile][lane] x 4 words, local row = 4 * unit + gate,
-// zero beyond the CTA's units and beyond column K.
-static std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int NW, int nkw, int MT)
-{
-    std::vector<uint32_t> f((size_t)ncta * NW * nkw * MT * 32 * 4, 0u);
-    size_t o = 0;
-    for (int c = 0; c < ncta; ++c) {
-        int u0, nu; unit_range_host(U, ncta, c, u0, nu);
-        auto wv = [&](int r, int k) -> uint32_t {
-            if (r >= 4 * nu || k >= K) return 0u;
-            return f32_to_bf16_rne(m[(size_t)((r & 3) * U + u0 + (r >> 2)) * K + k]);
-        };
-        for (int wp = 0; wp < NW; ++wp)
-            for (int i = 0; i < nkw; ++i)
-                for (int mt = 0; mt < MT; ++mt)
-                    for (int lane = 0; lane < 32; ++lane) {
-                        const int g = lane >> 2, p2 = (lane & 3) * 2;
-                        const int r0 = mt * 16 + g, r1 = r0 + 8;
-                        const int ka = (wp * nkw + i) * 16 + p2, kb = ka + 8;
-                        f[o++] = wv(r0, ka) | (wv(r0, ka + 1) << 16);
-                        f[o++] = wv(r1, ka) | (wv(r1, ka + 1) << 16);
-                        f[o++] = wv(r0, kb) | (wv(r0, kb + 1) << 16);
-                        f[o++] = wv(r1, kb) | (wv(r1, kb + 1) << 16);
-                    }
-    }
-    return f;
 }
 
 int hlstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int gate_hidden, int bidir, int dtype,
@@ -1016,6 +1025,35 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
             continue;
         }
+        if (h->use_csr_reg) {
+            RecurCsrArgs m;
+            memset(&m, 0, sizeof m);
+            m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
+            m.H = H; m.B = B; m.T = T; m.D = D; m.ncta_dir = h->ncta_dir; m.nsplit = nsplit;
+            m.kspan = h->csr_kspan; m.mt = h->csr_mt;
+            m.stamp_base = h->stamp_next;
+            h->stamp_next += (unsigned)T + 1u;
+            m.spin_limit = h->spin_limit;
+            m.withhold_cta = h->withhold_cta;
+            m.probe = B == 1 ? h->probe : 0;
+            for (int d = 0; d < D; ++d) { m.ent[d] = ly.csr_reg_ent[d]; m.rows[d] = ly.csr_reg_rows[d]; }
+            m.G = h->G;
+            m.g_split_stride = (long long)M * N;
+            const size_t so = (size_t)l * D * B * H;
+            m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
+            m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
+            m.y = l == L - 1 ? y : h->ybuf[l & 1];
+            m.xb_next = nullptr;
+            m.xch = h->xch;
+            m.status = h->status_dev;
+            const size_t smem = recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, B);
+            if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            e = launch_recur_csr_reg(m, h->csr_slots, h->csr_nw, smem, st);
+            ++h->last_launches;
+            if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+            if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));
+            continue;
+        }
         const RecurShape shp = recur_shape(h, B, l);
         if (h->use_mma) {
             RecurMmaArgs m;
@@ -1172,8 +1210,8 @@ int lstm_probe(lstm_handle *h, int parts_left_out)
 {
     if (!h) return LSTM_ERR_INVALID;
     if (parts_left_out < 0 || parts_left_out > 7) return fail(h, LSTM_ERR_INVALID, "probe mask %d outside 0..7", parts_left_out);
-    if (parts_left_out && (!h->use_mma || h->Hh))
-        return fail(h, LSTM_ERR_UNSUPPORTED, "only the register-resident recurrent kernel of an LSTM handle has probe modes");
+    if (parts_left_out && ((!h->use_mma && !h->use_csr_reg) || h->Hh))
+        return fail(h, LSTM_ERR_UNSUPPORTED, "only the register-resident recurrent kernels (dense and sparse) of an LSTM handle have probe modes");
     h->probe = parts_left_out;
     return LSTM_OK;
 }
@@ -1224,11 +1262,13 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
     const int tcb_at_max = (h->use_tcb && !h->Hh && h->max_B > 4 && h->max_B <= kTcMaxBatch &&
                             recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * h->max_B, 16), h->upc, h->max_B, (size_t)h->smem_optin - 256,
                                           h->tcb_pair ? 1 : 0, &ik, &is)) ? 1 : 0;
-    const int64_t vals[13] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->threads, (int64_t)shp.smem,
+    if (h->use_csr_reg) shp.smem = recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, h->max_B);
+    const int64_t vals[16] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->use_csr_reg ? h->csr_nw * 32 : h->threads, (int64_t)shp.smem,
                               rows_res, rows_str, (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches,
-                              h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0, tcb_at_max};
-    for (int i = 0; i < n && i < 13; ++i) out[i] = vals[i];
-    return 13;
+                              h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0, tcb_at_max,
+                              h->use_csr_reg ? 1 : 0, h->use_csr_reg ? h->csr_slots : 0, h->use_csr_reg ? h->csr_conflicts : 0};
+    for (int i = 0; i < n && i < 16; ++i) out[i] = vals[i];
+    return 16;
 }
 
 }  // extern "C"

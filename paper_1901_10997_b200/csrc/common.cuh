@@ -96,6 +96,47 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------------
+// Register-resident sparse recurrent kernel (bf16 weights, CSR execution).  Same CTA/unit partition,
+// exchange buffer and finishing role as the dense register-resident kernel.  Warp w of a CTA owns the
+// columns [w * kspan, (w + 1) * kspan) of h; inside the warp every lane owns up to two of the CTA's 4 * units
+// gate rows and keeps the surviving weights of those rows in that column range in registers for the whole
+// sequence, one 32-bit word each: {bf16 value : 16 | second-row flag : 1 | column inside the range : 15}.
+// A launch is compiled for E entry slots per lane; shorter lists are padded with zero words.
+// ---------------------------------------------------------------------------------------------------
+struct RecurCsrArgs {
+    int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
+    int H, B, T, D;
+    int ncta_dir;
+    int nsplit;
+    int kspan;                  // columns of h per warp (multiple of 32)
+    int hs_stride;              // floats of a warp's staging block: power of two >= rows per pass * kspan (set by the launcher)
+    int mt;                     // 16-row tiles that cover 4 * units per CTA (sets the pitch of the partial sums)
+    unsigned stamp_base;
+    long long spin_limit;
+    int withhold_cta;
+    int probe;                  // kProbe* bits, single-sequence calls only
+    const unsigned *ent[2];     // per direction [cta][warp][E][32 lanes] entry words
+    const unsigned *rows[2];    // per direction [cta][warp][32 lanes]: local rows of the lane's two lists
+                                //   (byte 0: first, byte 1: second; 0xff: none)
+    const float *G;
+    long long g_split_stride;
+    const float *h0, *c0;
+    float *hT, *cT;
+    float *y;
+    __nv_bfloat16 *xb_next;
+    long long xb_plane;
+    int xb_ld;
+    unsigned long long *xch;
+    int *status;
+};
+constexpr int kCsrRegMaxSlots16 = 64;    // entry slots per lane the kernel is built for with 16 warps ...
+constexpr int kCsrRegMaxSlots8 = 128;    // ... and with 8 warps (255 registers per thread)
+int recur_csr_reg_slots(int needed, int nw);     // smallest built slot count >= needed, or 0 when none is
+size_t recur_csr_reg_smem_bytes(int nw, int kspan, int mt, int upc, int B);
+cudaError_t recur_csr_reg_prepare(int slots, int nw, int max_smem);
+cudaError_t launch_recur_csr_reg(const RecurCsrArgs &a, int slots, int nw, size_t smem, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------
 // Batched recurrent kernel on tcgen05 (bf16 weights, dense, more than four batch rows).  The CTA's slice of
 // Wh sits in shared memory as K-major 128-byte-swizzled tiles of RA rows (4 * units per CTA rounded up to 8)
 // per 64 columns; h travels through global memory as bf16 planes [D][2 parities][64 rows][ldh] (row 2b = hi,

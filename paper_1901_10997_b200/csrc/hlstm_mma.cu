@@ -16,58 +16,14 @@
 //           published.
 // Batch rows are processed one after the other (two passes each).
 #include "common.cuh"
+#include "device_util.cuh"
 
 namespace lstm {
 namespace {
 
-__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
-{
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v)
-{
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ int ld_volatile_s32(const int *p)
-{
-    int v;
-    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ float ld_nc_early(const float *p)
-{
-    float v;
-    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
-__device__ __forceinline__ void bar_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4 &a, unsigned b0, unsigned b1)
-{
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
-}
 
-// logistic function and tanh z = 2 logistic(2z) - 1, each one exponential and one reciprocal
-__device__ __forceinline__ float ex2_fast(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float sigmoid_fast(float z) { return __fdividef(1.0f, 1.0f + ex2_fast(-1.4426950408889634f * z)); }
-__device__ __forceinline__ float tanh_fast(float z) { return fmaf(2.0f, __fdividef(1.0f, 1.0f + ex2_fast(-2.8853900817779268f * z)), -1.0f); }
 
-__device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
-{
-    const int base = H / nc, rem = H % nc;
-    n = base + (c < rem ? 1 : 0);
-    u0 = c * base + (c < rem ? c : rem);
-}
 
 constexpr int kPoll = 4;
 constexpr int kMaxSplit = 4;

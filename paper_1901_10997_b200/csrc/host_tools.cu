@@ -3,7 +3,9 @@
 // next layer's input weights (paper, Section 5.2: batch normalisation between recurrent layers, which at
 // inference time is a fixed scale and shift per feature).
 #include "../../include/lstm_b200.h"
+#include "csr_pack.h"
 
+#include <algorithm>
 #include <cmath>
 #include <limits>
 #include <vector>
@@ -74,3 +76,27 @@ int lstm_fold_input_affine(const float *wx, const float *b, int rows, int cols, 
 }
 
 }  // extern "C"
+
+
+// The create-time layout of one pruned recurrent matrix for the register-resident sparse kernel, exposed so
+// that it can be inspected without a GPU (see the header).
+extern "C" int lstm_csr_lane_layout(const int32_t *rowptr, const int32_t *col, const float *val, int hidden, int ctas,
+                                    int warps, int kspan, int slots, uint32_t *entries, uint32_t *rows, int *longest,
+                                    long long *conflict_wavefronts)
+{
+    if (!rowptr || hidden < 1 || ctas < 1 || ctas > hidden || (warps != 8 && warps != 16) || kspan < 32 || (kspan % 32) != 0 ||
+        kspan * 4 > 0x7ffc || (long long)kspan * warps < hidden || slots < 0)
+        return LSTM_ERR_INVALID;
+    if ((hidden + ctas - 1) / ctas > warps) return LSTM_ERR_UNSUPPORTED;      // more than 4 * warps rows per CTA
+    if (rowptr[4 * hidden] > 0 && (!col || !val)) return LSTM_ERR_INVALID;
+    lstm::CsrLaneLists lists;
+    lstm::csr_lane_lists(rowptr, col, val, hidden, ctas, warps, kspan, lists);
+    if (longest) *longest = lists.longest;
+    if (rows) std::copy(lists.rows.begin(), lists.rows.end(), rows);
+    if (entries) {
+        if (slots < lists.longest) return LSTM_ERR_INVALID;
+        const std::vector<unsigned> packed = lstm::csr_pack_slots(lists, ctas, warps, slots, kspan, conflict_wavefronts);
+        std::copy(packed.begin(), packed.end(), entries);
+    }
+    return LSTM_OK;
+}

@@ -14,34 +14,12 @@
 // costs a single L2 round trip after the last producer's store and needs no separate barrier.
 // Every wait is bounded: when it expires the CTA records a timeout status and leaves.
 #include "common.cuh"
+#include "device_util.cuh"
 
 namespace lstm {
 namespace {
 
-__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
-{
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v)
-{
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ int ld_volatile_s32(const int *p)
-{
-    int v;
-    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
 
-// read-only load that the compiler may not sink towards its use: issued before a wait, consumed after it
-__device__ __forceinline__ float ld_nc_early(const float *p)
-{
-    float v;
-    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
-    return v;
-}
 
 __device__ __forceinline__ float sigmoid_f(float z) { return 1.0f / (1.0f + expf(-z)); }
 
@@ -81,12 +59,6 @@ __device__ __forceinline__ AT warp_reduce_multi(AT (&v)[V], int lane)
     return v[0];
 }
 
-__device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
-{
-    const int base = H / nc, rem = H % nc;
-    n = base + (c < rem ? 1 : 0);
-    u0 = c * base + (c < rem ? c : rem);
-}
 
 // eight weights of one row at vector index v8 -> fp32
 __device__ __forceinline__ void load_w8(const __nv_bfloat16 *row, int v8, float (&w)[8])

@@ -27,77 +27,14 @@
 // between two barriers and two partial-sum buffers).  Every wait on another CTA is bounded: when it
 // expires the CTA records a timeout status, stops waiting for the rest of the launch and runs to the end.
 #include "common.cuh"
+#include "device_util.cuh"
 
 namespace lstm {
 namespace {
 
-__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
-{
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_relaxed_u64(unsigned long long *p, unsigned long long v)
-{
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ int ld_volatile_s32(const int *p)
-{
-    int v;
-    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-// read-only load that the compiler may not sink towards its use: issued early, consumed a step later
-__device__ __forceinline__ float ld_nc_early(const float *p)
-{
-    float v;
-    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
-    return v;
-}
-// 16-byte asynchronous copy global -> shared through L2 only (never a stale L1 line)
-__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gsrc)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all()
-{
-    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
-__device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
-__device__ __forceinline__ void bar_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
-// D += A (16x16, row) * B (16x8, col), bf16 inputs, fp32 accumulation
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4 &a, unsigned b0, unsigned b1)
-{
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
-}
 
-// gate functions from the fast exponential: absolute error of a few 1e-7, far inside the 2e-2 bound of
-// the bf16 storage type
-// Both gate functions as one expression, sc / (1 + 2^(-k log2(e) z)) + of: the logistic function with
-// (k, sc, of) = (1, 1, 0) and tanh z = 2 logistic(2z) - 1 with (2, 2, -1).  One exponential and one
-// reciprocal on the path from the summed pre-activation to the published h, and no select between two
-// evaluated functions.
-__device__ __forceinline__ float ex2_fast(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float gate_fast(float z, float neg_k_log2e, float sc, float of)
-{
-    return fmaf(sc, __fdividef(1.0f, 1.0f + ex2_fast(neg_k_log2e * z)), of);
-}
-__device__ __forceinline__ float tanh_fast(float z) { return gate_fast(z, -2.0f * 1.4426950408889634f, 2.0f, -1.0f); }
 
-__device__ __forceinline__ void unit_range(int H, int nc, int c, int &u0, int &n)
-{
-    const int base = H / nc, rem = H % nc;
-    n = base + (c < rem ? 1 : 0);
-    u0 = c * base + (c < rem ? c : rem);
-}
 
 constexpr int kPoll = 4;      // exchange words a lane keeps in flight per polling round
 constexpr int kMaxSplit = 4;  // split-K planes of the projection output (the projection plans at most 4)
