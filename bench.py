@@ -50,6 +50,8 @@ FALLBACK_HBM_GBS = 6650.0
 LEGS = [("cfg2_b20", "cfg2_b20", 20), ("cfg5_b16", "cfg5_b16", 3), ("cfg5_b1", "cfg5", 5),
         ("cfg4_d10_dense_with_zeros", "cfg4_10", 20), ("cfg4_d10_csr", "cfg4_10_csr", 20),
         ("cfg4_d05_dense_with_zeros", "cfg4_05", 20), ("cfg4_d05_csr", "cfg4_05_csr", 20),
+        ("cfg2_units_pruned_1197_compacted", "cfg2_rc", 20), ("cfg2_units_pruned_1197_zeros_kept", "cfg2_rc_zeros", 20),
+        ("cfg2_units_pruned_1197_b20_compacted", "cfg2_rc_b20", 10), ("cfg2_units_pruned_1197_b20_zeros_kept", "cfg2_rc_b20_zeros", 10),
         ("cfg1_fp32_b20", "cfg1", 20)]
 
 
@@ -62,6 +64,12 @@ def pick_workload(name: str):
         "cfg4_05": (wl.config4(0.05), "dense"),
         "cfg4_10_csr": (wl.config4(0.10), "csr"),
         "cfg4_05_csr": (wl.config4(0.05), "csr"),
+        # row/column pruning (Section 4.2, Table 1 step (b)): 303 of 1500 hidden units per layer removed; run on the
+        # surviving units (compacted) or with the zeros kept in the 1500-wide model
+        "cfg2_rc": (wl.config2_units_pruned(1), "dense"),
+        "cfg2_rc_zeros": (wl.config2_units_pruned(1), "dense"),
+        "cfg2_rc_b20": (wl.config2_units_pruned(20), "dense"),
+        "cfg2_rc_b20_zeros": (wl.config2_units_pruned(20), "dense"),
         "cfg5": (wl.config5(1), "dense"),
         "cfg5_b16": (wl.config5(16), "dense"),
         # H-LSTM cell (one ReLU hidden layer of the cell's width inside each gate), the paper's own models:
@@ -104,7 +112,12 @@ def measured_traffic(kernel: str, workload: str, source: str):
 
 
 def make_inputs(w: wl.Workload, mode: str):
-    return wl.make_hlstm(w, w.hidden) if mode == "hlstm" else wl.make(w)
+    if mode == "hlstm":
+        return wl.make_hlstm(w, w.hidden)
+    weights, x = wl.make(w)
+    if w.name.startswith("cfg2_units_pruned"):
+        weights, _removed = wl.prune_units(w, weights, 1197)
+    return weights, x
 
 
 def oracle_forward(w: wl.Workload, mode: str, weights, xs):
@@ -361,8 +374,20 @@ class GpuCase:
             self.model = pkg.HLSTM(self.weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, gate_hidden=w.hidden,
                                    bidir=w.bidir, dtype=w.dtype, max_T=w.T, max_B=w.B)
         else:
-            self.model = pkg.LSTM(self.weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir,
-                                  dtype=w.dtype, exec_mode=self.mode, max_T=w.T, max_B=w.B)
+            keep_zeros = workload_name.endswith("_zeros")
+            force = workload_name.startswith("cfg2_rc")
+            old = os.environ.get("LSTM_B200_COMPACT")
+            if force:
+                os.environ["LSTM_B200_COMPACT"] = "0" if keep_zeros else "1"
+            try:
+                self.model = pkg.LSTM(self.weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir,
+                                      dtype=w.dtype, exec_mode=self.mode, max_T=w.T, max_B=w.B)
+            finally:
+                if force:
+                    if old is None:
+                        os.environ.pop("LSTM_B200_COMPACT", None)
+                    else:
+                        os.environ["LSTM_B200_COMPACT"] = old
         self.dev = dev
         self.flush_buf = flush_buf
         self.xd = torch.from_numpy(self.x).to(dev)
@@ -603,6 +628,7 @@ def run_legs(torch, pkg, dev, flush_buf, cache, peak, peak_kind):
                 "gpu_launches": int(case.model.info()["launches_per_forward"] * steps),
                 "kernel_ms_per_forward": {"stage": stage_ms / nk, "projection": proj_ms / nk, "recurrence": rec_ms / nk},
                 "roofline": case.roofline(rec_ms, rec_n, peak, peak_kind),
+                "library": case.model.info(),
                 "clocks": clocks.summary(),
                 "wall_s": None,
             }

@@ -103,6 +103,19 @@ typedef struct {
  *                   = mma   no batched tensor-core recurrence (batches above four run as passes of four)
  *                   = tc1   batched tensor-core recurrence without cluster pairs
  *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
+ *   LSTM_B200_COMPACT = 0   keep row/column-pruned units as explicit zeros, = 1 always run on the surviving units
+ *                           (unset: handles with max_B >= 5 compact, smaller ones keep the zeros; see below)
+ * Row/column-pruned stacks (Section 4.2, Algorithm 1: whole rows and columns of the gate matrices are zero).
+ * lstm_create (for max_B >= 5, or when LSTM_B200_COMPACT=1) looks for hidden units that read nothing and are read by nobody: all four gate rows zero in Wx and
+ * Wh, the unit's column of Wh zero and, below the last layer, its column of every next-layer Wx zero.  If every
+ * (layer, direction) has such units, the forward pass runs on the surviving units only, at the compact width
+ * Hc = the largest number of survivors of any matrix (what the paper's pruning buys on a GPU: a smaller dense
+ * model); the removed units' outputs and final states follow from their biases and c0 in closed form
+ * (constant gates) and are written beside the survivors', so y, hT and cT keep the full width and the result
+ * equals the dense-with-zeros one.  Such a handle costs one small extra kernel per call (two when h0 or c0 is
+ * given) and does not serve lstm_input_projection.  Handles for up to four sequences keep the zeros by default:
+ * their step is bound by the exchange latency, not by the width, and the extra kernel would cost more than the
+ * narrower model saves.
  *   LSTM_B200_SPIN_LIMIT = <clock ticks>  bound of every device-side wait (default about two seconds)
  */
 LSTM_API int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int bidir, int dtype,
@@ -224,7 +237,10 @@ LSTM_API int lstm_probe(lstm_handle *h, int parts_left_out);
  * register-resident kernel (passes of four sequences) otherwise,
  * [13] 1 if a CSR handle runs the register-resident sparse kernel (bf16 storage, at most 16 units per CTA,
  * lane lists short enough for registers), 0 for the shared-memory CSR kernel, [14] its entry slots per lane,
- * [15] shared-memory wavefronts per step and CTA that its gathers lose to bank conflicts (worst CTA).
+ * [15] shared-memory wavefronts per step and CTA that its gathers lose to bank conflicts (worst CTA),
+ * [16] the compact width when the handle runs a row/column-pruned stack on its surviving units only (0: it does
+ * not; then [0]..[15] describe the handle itself, otherwise the inner handle of that width), [17] the number
+ * of (layer, direction, unit) triples removed.
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 

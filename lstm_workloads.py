@@ -90,6 +90,42 @@ def config5_width(H: int, B: int = 16) -> Workload:
     return Workload(f"ds2_sweep_H{H}_B{B}", 5, True, 1312, H, 400, B, "bf16", 1.0 / math.sqrt(H), seed=_seed(5, H))
 
 
+def config2_units_pruned(B: int = 1) -> Workload:
+    """Large language-model shape after row/column pruning (paper, Section 4.2 and Table 1 step (b): hidden
+    width 1500 pruned to 1197): the same two layers of width 1500, with 303 hidden units per layer whose rows
+    and columns are zero (see ``prune_units``)."""
+    return Workload(f"cfg2_units_pruned_B{B}", 2, False, 1500, 1500, 35, B, "bf16", 0.04, seed=_seed(2, 1197))
+
+
+def prune_units(w: Workload, weights, keep: int, seed_offset: int = 11):
+    """Row/column pruning at the level of whole hidden units, the structure Algorithm 1 of the paper leaves
+    behind: for every (layer, direction) a seeded random set of ``hidden - keep`` units loses all its incoming
+    weights (the four gate rows of ``wx`` and ``wh``) and all its outgoing ones (its column of ``wh`` and of the
+    next layer's ``wx``).  Biases stay.  Returns (weights with the zeros written in, removed) where
+    ``removed[layer * dirs + d]`` is the sorted array of pruned units.  No arithmetic of the model happens here."""
+    rng = np.random.Generator(np.random.PCG64(w.seed + seed_offset))
+    H, D = w.hidden, w.dirs
+    out = [{k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in e.items()} for e in weights]
+    removed = []
+    for l in range(w.layers):
+        for d in range(D):
+            gone = np.sort(rng.choice(H, size=H - keep, replace=False))
+            removed.append(gone)
+            e = out[l * D + d]
+            rows = (np.arange(4)[:, None] * H + gone[None, :]).ravel()
+            e["wx"][rows, :] = 0.0
+            e["wh"][rows, :] = 0.0
+            e["wh"][:, gone] = 0.0
+            if l + 1 < w.layers:
+                for d2 in range(D):
+                    out[(l + 1) * D + d2]["wx"][:, d * H + gone] = 0.0
+    for e in out:
+        for m, name in (("mask_x", "wx"), ("mask_h", "wh")):
+            if m in e:
+                e[m] = (e[m].astype(bool) & (e[name] != 0)).astype(np.uint8)
+    return out, removed
+
+
 def round_to_bf16(a: np.ndarray) -> np.ndarray:
     """float32 -> nearest-even bfloat16 -> float32 (finite inputs)."""
     a = np.ascontiguousarray(a, dtype=np.float32)

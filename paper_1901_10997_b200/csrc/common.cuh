@@ -215,6 +215,26 @@ cudaError_t hlstm_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_hlstm_mma(const HlstmArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------------
+// Row/column-pruned stacks: moving states and outputs between the full width H and the compact width Hc of the
+// surviving units, and the closed-form recurrence of the removed ones.
+// ---------------------------------------------------------------------------------------------------
+struct CompactArgs {
+    int L, D, H, Hc, T, B;
+    const int *cmap;            // [L*D][Hc]: unit of the full model behind compact unit jc
+    int n_removed;
+    const int *rem_idx;         // [n_removed][2]: {layer * D + direction, unit}
+    const float *rem_bias;      // [n_removed][4]: b_i, b_f, b_g, b_o of the removed unit
+    const float *h0, *c0;       // caller's [L*D][B][H] or nullptr
+    float *h0c, *c0c;           // compact [L*D][B][Hc]
+    const float *yc;            // compact [T][B][D*Hc]
+    const float *hTc, *cTc;     // compact [L*D][B][Hc]
+    float *y;                   // caller's [T][B][D*H]
+    float *hT, *cT;             // caller's [L*D][B][H] or nullptr
+};
+cudaError_t launch_compact_gather(const CompactArgs &a, cudaStream_t st);
+cudaError_t launch_compact_scatter(const CompactArgs &a, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------
 // Input staging and projection
 // ---------------------------------------------------------------------------------------------------
 // x fp32 [M][K] -> two bf16 planes [M][ld]: hi = bf16(x), lo = bf16(x - hi) at xb + plane
