@@ -19,6 +19,7 @@ Other modes:
     --impl reference     time the fp64 CPU oracle on the same workload (host cores only)
     --sweep              latency vs hidden size (H = 128..2048 step 8) with the LHP analysis
     --matmul-sweep       dense (tensor-core) vs sparse (CSR) matrix product at batch 16, d = 128..2048
+    --wave-sweep         layer-wavefront kernel vs one launch per layer over H (2 layers, T = 35, batch 1)
     --workload NAME      cfg1 | cfg2 | cfg2_b20 | cfg4_10 | cfg4_05 | cfg4_10_csr | cfg4_05_csr |
                          cfg5 | cfg5_b16 | hlstm_ptb | hlstm_ds2 (default cfg2)
     --no-legs            headline workload only
@@ -766,6 +767,63 @@ def run_matmul_sweep(args):
     print(json.dumps(summary))
 
 
+def run_wave_sweep(args):
+    """Layer-wavefront kernel against one launch per layer on the two-layer language-model shape (input = hidden
+    = H, T = 35, batch 1, bf16 weights): microseconds per sequence for both, the same handle settings otherwise.
+    Timed like the hidden-size sweep (`us_cold`: L2 flushed, one call per event pair; `us_warm`: calls back to
+    back inside one pair)."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    dev = torch.device("cuda", 0)
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    outdir = Path(args.out)
+    outdir.mkdir(parents=True, exist_ok=True)
+    sizes = [int(s) for s in args.sweep_sizes.split(",")] if args.sweep_sizes else [128, 200, 256, 384, 512, 640, 768, 896, 1000, 1024]
+    layers = args.wave_layers
+    rows = []
+    for H in sizes:
+        w = wl.Workload(f"wave_sweep_L{layers}_H{H}", layers, False, H, H, 35, args.wave_batch, "bf16", 1.0 / np.sqrt(H), seed=wl.SEED_BASE + 7 * H + layers)
+        weights, x = wl.make(w)
+        xd = torch.from_numpy(x).to(dev)
+        out = (torch.empty((w.T, w.B, H), device=dev), torch.empty((layers, w.B, H), device=dev), torch.empty((layers, w.B, H), device=dev))
+        row = {"H": H, "layers": layers, "B": w.B}
+        old = os.environ.get("LSTM_B200_WAVE")
+        try:
+            for label, env in (("wavefront", "1"), ("per_layer", "0")):
+                os.environ["LSTM_B200_WAVE"] = env
+                m = pkg.LSTM(weights, layers=layers, in_dim=H, hidden=H, dtype="bf16", max_T=w.T, max_B=w.B)
+                info = m.info()
+                if label == "wavefront" and not info["layer_wavefront"]:
+                    m.close()
+                    row["wavefront_served"] = False
+                    continue
+                fn = lambda: m.forward(xd, out=out)
+                ms = time_steps(fn, args.steps, max(args.warmup, 3), flush_buf, torch)
+                m.check()
+                cold = trimmed_mean(ms)
+                warm = time_back_to_back(fn, max(1, int(np.ceil(0.2 / max(cold, 1e-4)))), 9, torch)
+                m.check()
+                row[label + "_us_cold"] = cold * 1e3
+                row[label + "_us_warm"] = warm * 1e3
+                row[label + "_launches"] = m.info()["launches_per_forward"]
+                if args.sweep_parity:
+                    import oracle
+                    ref = oracle.forward(weights, x, layers=layers, bidir=False, hidden=H)
+                    row[label + "_err"] = max(wl.rel_err(g.cpu().numpy(), r)[1] for g, r in zip(out, ref))
+                m.close()
+        finally:
+            if old is None:
+                os.environ.pop("LSTM_B200_WAVE", None)
+            else:
+                os.environ["LSTM_B200_WAVE"] = old
+        rows.append(row)
+        print(json.dumps(row), file=sys.stderr, flush=True)
+    (outdir / f"wave_sweep_L{layers}_B{args.wave_batch}.json").write_text(json.dumps({"steps": args.steps, "points": rows}, indent=1))
+    print(json.dumps({"points": len(rows),
+                      "wavefront_faster_cold": [r["H"] for r in rows if r.get("wavefront_us_cold", 1e9) < r.get("per_layer_us_cold", 0)],
+                      "wavefront_faster_warm": [r["H"] for r in rows if r.get("wavefront_us_warm", 1e9) < r.get("per_layer_us_warm", 0)]}))
+
+
 def _free_port():
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
@@ -814,13 +872,16 @@ def main():
     ap.add_argument("--no-legs", action="store_true")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--matmul-sweep", action="store_true")
+    ap.add_argument("--wave-sweep", action="store_true")
+    ap.add_argument("--wave-layers", type=int, default=2)
+    ap.add_argument("--wave-batch", type=int, default=1)
     ap.add_argument("--sweep-sizes", default="")
     ap.add_argument("--sweep-shape", default="cfg3", choices=["cfg3", "ds2"])
     ap.add_argument("--sweep-parity", action="store_true")
     ap.add_argument("--out", default=str(ROOT / "bench_out"))
     ap.add_argument("--replica-check", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.sweep or args.matmul_sweep):
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.sweep or args.matmul_sweep or args.wave_sweep):
         raise SystemExit(spawn_replicas(args))
     if args.replica_check:
         run_replica_check(args)
@@ -830,6 +891,8 @@ def main():
         run_sweep(args)
     elif args.matmul_sweep:
         run_matmul_sweep(args)
+    elif args.wave_sweep:
+        run_wave_sweep(args)
     else:
         run_gpu(args)
 

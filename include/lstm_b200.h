@@ -102,6 +102,7 @@ typedef struct {
  *   LSTM_B200_RECUR = simt  shared-memory recurrent kernel instead of the register-resident one (bf16 dense or CSR)
  *                   = mma   no batched tensor-core recurrence (batches above four run as passes of four)
  *                   = tc1   batched tensor-core recurrence without cluster pairs
+ *   LSTM_B200_WAVE  = 0     one launch per layer even where the layer-wavefront kernel would serve the stack
  *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
  *   LSTM_B200_COMPACT = 0   keep row/column-pruned units as explicit zeros, = 1 always run on the surviving units
  *                           (unset: handles with max_B >= 5 compact, smaller ones keep the zeros; see below)
@@ -240,7 +241,9 @@ LSTM_API int lstm_probe(lstm_handle *h, int parts_left_out);
  * [15] shared-memory wavefronts per step and CTA that its gathers lose to bank conflicts (worst CTA),
  * [16] the compact width when the handle runs a row/column-pruned stack on its surviving units only (0: it does
  * not; then [0]..[15] describe the handle itself, otherwise the inner handle of that width), [17] the number
- * of (layer, direction, unit) triples removed.
+ * of (layer, direction, unit) triples removed, [18] 1 if calls with up to four sequences run the layer-wavefront
+ * kernel (unidirectional bf16 dense stacks of 2 to 4 layers whose slices fit on-chip with the SMs split between
+ * the layers: all layers in one launch, layer l on timestep t beside layer l-1 on t+1).
  */
 LSTM_API int lstm_info(const lstm_handle *h, int64_t *out, int n);
 

@@ -162,7 +162,7 @@ def lstm_info(handle):
             "proj_splits", "proj_tensor_core", "launches_per_forward", "recur_register_resident",
             "col_tiles_in_registers", "col_tiles_in_smem", "recur_batched_tensor_core",
             "recur_csr_register_resident", "csr_slots_per_lane", "csr_bank_conflict_wavefronts",
-            "compact_hidden", "units_removed"]
+            "compact_hidden", "units_removed", "layer_wavefront"]
     return {k: int(out[i]) for i, k in enumerate(keys[:n])}
 
 

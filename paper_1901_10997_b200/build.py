@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "liblstm_b200.so"
 INCLUDE = PKG.parent / "include"
-SOURCES = ["api.cu", "recur.cu", "proj_simt.cu", "proj_tc.cu", "noalloc.cu", "recur_mma.cu", "hlstm_mma.cu", "recur_tc.cu", "host_tools.cu", "recur_csr.cu", "csr_pack.cu", "compact.cu"]
+SOURCES = ["api.cu", "recur.cu", "proj_simt.cu", "proj_tc.cu", "noalloc.cu", "recur_mma.cu", "hlstm_mma.cu", "recur_tc.cu", "host_tools.cu", "recur_csr.cu", "csr_pack.cu", "compact.cu", "recur_wave.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false"]
 

@@ -92,6 +92,11 @@ struct lstm_handle {
     std::vector<int> ev_kind;
     int ev_used = 0;
     int last_launches = 0;
+    // layer-wavefront kernel (unidirectional stacks, up to four sequences): CTAs per layer, units per CTA, tiling
+    bool use_wave = false;
+    int wave_ncta = 0, wave_upc = 0, wave_mt = 0, wave_nkr = 0, wave_nkw[kMaxWaveLayers] = {0, 0, 0, 0}, wave_nkw_max = 0;
+    uint4 *wave_frag[kMaxWaveLayers] = {nullptr, nullptr, nullptr, nullptr};
+    unsigned long long *wave_xch = nullptr; size_t wave_xch_words = 0;
     // row/column-pruned stacks: the forward pass runs on an inner handle over the surviving units (width Hc)
     lstm_handle *inner = nullptr;
     int Hc = 0, n_removed = 0;
@@ -377,6 +382,33 @@ std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int
     return f;
 }
 
+// Tiling of the layer-wavefront kernel, or use_wave = false when the stack does not qualify: one direction, two
+// to four layers, bf16 dense, at most 16 units per CTA with the SMs split evenly between the layers, and the
+// widest layer's slice (4 * units rows by 2H columns) inside registers + shared memory.
+void plan_wave(lstm_handle *h)
+{
+    h->use_wave = false;
+    if (h->D != 1 || h->L < 2 || h->L > kMaxWaveLayers || h->dtype != LSTM_BF16W_F32S || h->exec_mode != LSTM_DENSE || h->Hh) return;
+    const char *env = getenv("LSTM_B200_WAVE");
+    if (env && strcmp(env, "0") == 0) return;
+    const int H = h->H;
+    const int n = std::max(1, std::min(h->sm_count / h->L, H));
+    const int upc = (H + n - 1) / n;
+    if (upc > 16) return;
+    const int mt = (4 * upc + 15) / 16;
+    const int need0 = ((H + 15) / 16 + 15) / 16, need1 = ((2 * H + 15) / 16 + 15) / 16;
+    const int cap = kWaveTileCap / mt;
+    int nkr = 0;
+    for (int c = 2; c <= 8; c += 2)
+        if (c <= cap && (nkr == 0 || nkr < need1)) nkr = c;
+    if (nkr == 0 || !recur_wave_shape_ok(mt, nkr)) return;
+    const int nkw0 = std::max(need0, nkr), nkw1 = std::max(need1, nkr);
+    if (recur_wave_smem_bytes(mt, nkr, nkw1, upc, std::min(h->max_B, 4)) > (size_t)h->smem_optin - 64) return;
+    h->use_wave = true;
+    h->wave_ncta = n; h->wave_upc = upc; h->wave_mt = mt; h->wave_nkr = nkr; h->wave_nkw_max = nkw1;
+    for (int l = 0; l < h->L; ++l) h->wave_nkw[l] = l == 0 ? nkw0 : nkw1;
+}
+
 void free_all(lstm_handle *h)
 {
     for (auto &ly : h->layers) {
@@ -386,6 +418,8 @@ void free_all(lstm_handle *h)
     }
     cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
     cudaFree(h->ybuf[0]); cudaFree(h->ybuf[1]); cudaFree(h->xch); cudaFree(h->rxch); cudaFree(h->hplanes); cudaFree(h->tcb_flags); cudaFree(h->status_dev);
+    for (int l = 0; l < kMaxWaveLayers; ++l) cudaFree(h->wave_frag[l]);
+    cudaFree(h->wave_xch);
     cudaFree(h->cmap); cudaFree(h->rem_idx); cudaFree(h->rem_bias);
     cudaFree(h->ch0); cudaFree(h->cc0); cudaFree(h->cy); cudaFree(h->chT); cudaFree(h->ccT);
     cudaFree(h->hx); cudaFree(h->hy); cudaFree(h->hh0); cudaFree(h->hc0); cudaFree(h->hhT); cudaFree(h->hcT);
@@ -468,6 +502,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
     plan_mma(h);
+    plan_wave(h);
     if (csr && bf16) {
         // the register-resident sparse kernel: at most 16 units per CTA (warp w finishes unit w, a lane owns at
         // most two of the 4 * units rows); the entry slots per lane are known once every matrix has been laid out
@@ -551,6 +586,8 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                 snprintf(name, sizeof name, "wx[layer %d, dir %d]", l, d);
                 rc = matrix_to_dense(h, 4 * H, ly.in_l, src.wx, src.mask_x, src.wx_rowptr, src.wx_col, src.wx_val, m, name);
                 if (rc) break;
+                std::vector<float> wave_x;
+                if (h->use_wave && l > 0) wave_x = m;                 // the wavefront kernel folds Wx of the upper layers into the step
                 for (int q = 0; q < 4; ++q)
                     for (int j = 0; j < H; ++j) {
                         const float *srow = m.data() + (size_t)(q * H + j) * ly.in_l;
@@ -561,6 +598,25 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                 snprintf(name, sizeof name, "wh[layer %d, dir %d]", l, d);
                 rc = matrix_to_dense(h, 4 * H, H, src.wh, src.mask_h, src.wh_rowptr, src.wh_col, src.wh_val, m, name);
                 if (rc) break;
+                if (h->use_wave) {
+                    // layer 0: Wh alone; above: [Wx | Wh] side by side, 2H columns
+                    std::vector<float> cat;
+                    const float *src_m = m.data();
+                    int Kw = H;
+                    if (l > 0) {
+                        Kw = 2 * H;
+                        cat.resize((size_t)4 * H * Kw);
+                        for (int r = 0; r < 4 * H; ++r) {
+                            memcpy(cat.data() + (size_t)r * Kw, wave_x.data() + (size_t)r * H, sizeof(float) * H);
+                            memcpy(cat.data() + (size_t)r * Kw + H, m.data() + (size_t)r * H, sizeof(float) * H);
+                        }
+                        src_m = cat.data();
+                    }
+                    const std::vector<uint32_t> f = pack_fragments(src_m, H, Kw, h->wave_ncta, 16, h->wave_nkw[l], h->wave_mt);
+                    rc = upload(h, (uint32_t **)&h->wave_frag[l], f.data(), f.size() * 4, st, "wavefront weight fragments");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                    if (rc) break;
+                }
                 const size_t n = (size_t)H * 4 * h->Hp8;
                 if (h->use_mma) {
                     const std::vector<uint32_t> f = pack_fragments(m.data(), H, H, h->ncta_dir, h->mma_nw, h->mma_nkr + h->mma_nks, h->mma_mt);
@@ -709,6 +765,12 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         if (rc == LSTM_OK) rc = dev_alloc(h, &h->tcb_flags, (size_t)D * h->ncta_dir * sizeof(unsigned), true, st, "stamps");
     }
     if (rc == LSTM_OK) rc = dev_alloc(h, &h->status_dev, sizeof(int), true, st, "status word");
+    if (rc == LSTM_OK && h->use_wave) {
+        h->wave_xch_words = (size_t)layers * max_T * std::min(max_B, 4) * H;
+        rc = dev_alloc(h, &h->wave_xch, h->wave_xch_words * 8, true, st, "wavefront exchange buffer");
+        if (rc == LSTM_OK && recur_wave_prepare(h->wave_mt, h->wave_nkr, h->smem_optin - 64) != cudaSuccess)
+            rc = fail(h, LSTM_ERR_CUDA, "wavefront kernel set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
     if (rc == LSTM_OK) {
         cudaError_t e = h->use_csr_reg ? recur_csr_reg_prepare(h->csr_slots, h->csr_nw, h->smem_optin - 64)
                             : csr ? recur_csr_prepare(h->smem_optin - 64)
@@ -1124,7 +1186,35 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         if (cudaMemsetAsync(h->xch, 0, h->xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->rxch && cudaMemsetAsync(h->rxch, 0, h->rxch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         if (h->tcb_flags && cudaMemsetAsync(h->tcb_flags, 0, (size_t)D * h->ncta_dir * sizeof(unsigned), st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
+        if (h->wave_xch && cudaMemsetAsync(h->wave_xch, 0, h->wave_xch_words * 8, st) != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "exchange reset failed");
         h->stamp_next = 1;
+    }
+
+    if (h->use_wave && B <= 4) {
+        // all layers in one launch: layer 0's projection for all timesteps, then the wavefront kernel
+        int nsplit = 1;
+        { const int prc = run_projection(h, 0, x, x, M, D * 4 * H, &nsplit, st); if (prc != LSTM_OK) return prc; }
+        RecurWaveArgs m;
+        memset(&m, 0, sizeof m);
+        m.L = L; m.H = H; m.B = B; m.T = T; m.ncta_layer = h->wave_ncta; m.nsplit = nsplit;
+        for (int l = 0; l < L; ++l) { m.nkw[l] = h->wave_nkw[l]; m.wfrag[l] = h->wave_frag[l]; m.bias[l] = h->layers[l].bias; }
+        m.nkw_max = h->wave_nkw_max;
+        m.stamp_base = h->stamp_next;
+        h->stamp_next += (unsigned)T + 1u;
+        m.spin_limit = h->spin_limit;
+        m.withhold_cta = h->withhold_cta;
+        m.G = h->G;
+        m.g_split_stride = (long long)M * 4 * H;
+        m.h0 = h0; m.c0 = c0; m.hT = hT; m.cT = cT; m.y = y;
+        m.xch = h->wave_xch;
+        m.status = h->status_dev;
+        const size_t smem = recur_wave_smem_bytes(h->wave_mt, h->wave_nkr, h->wave_nkw_max, h->wave_upc, B);
+        if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        e = launch_recur_wave(m, h->wave_mt, h->wave_nkr, smem, st);
+        ++h->last_launches;
+        if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
+        if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "wavefront launch failed: %s", cudaGetErrorString(e));
+        return LSTM_OK;
     }
 
     for (int l = 0; l < L; ++l) {
@@ -1464,12 +1554,12 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
                             recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * h->max_B, 16), h->upc, h->max_B, (size_t)h->smem_optin - 256,
                                           h->tcb_pair ? 1 : 0, &ik, &is)) ? 1 : 0;
     if (h->use_csr_reg) shp.smem = recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, h->max_B);
-    const int64_t vals[18] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->use_csr_reg ? h->csr_nw * 32 : h->threads, (int64_t)shp.smem,
+    const int64_t vals[19] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->use_csr_reg ? h->csr_nw * 32 : h->threads, (int64_t)shp.smem,
                               rows_res, rows_str, (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches,
                               h->use_mma ? 1 : 0, h->use_mma ? h->mma_nkr : 0, h->use_mma ? h->mma_nks : 0, tcb_at_max,
-                              h->use_csr_reg ? 1 : 0, h->use_csr_reg ? h->csr_slots : 0, h->use_csr_reg ? h->csr_conflicts : 0, 0, 0};
-    for (int i = 0; i < n && i < 18; ++i) out[i] = vals[i];
-    return 18;
+                              h->use_csr_reg ? 1 : 0, h->use_csr_reg ? h->csr_slots : 0, h->use_csr_reg ? h->csr_conflicts : 0, 0, 0, h->use_wave ? 1 : 0};
+    for (int i = 0; i < n && i < 19; ++i) out[i] = vals[i];
+    return 19;
 }
 
 }  // extern "C"

@@ -96,6 +96,38 @@ cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------------
+// Layer-wavefront recurrent kernel (unidirectional stacks of 2 to 4 layers, bf16 dense, up to four sequences).
+// CTAs [l * ncta_layer, (l + 1) * ncta_layer) run layer l.  Layer 0's matrix is Wh_0 [4H x H]; layer l >= 1's
+// is [Wx_l | Wh_l] [4H x 2H] acting on [h^{l-1}_t ; h^l_{t-1}].  Fragment layout as in RecurMmaArgs with
+// nkw[l] column tiles per warp (the first NKR in registers).
+// ---------------------------------------------------------------------------------------------------
+constexpr int kMaxWaveLayers = 4;
+constexpr int kWaveTileCap = 16;     // MT * NKR limit (128 registers per thread at 16 warps, no spills)
+struct RecurWaveArgs {
+    int L, H, B, T;
+    int ncta_layer;
+    int nsplit;                 // partial planes of layer 0's projection output
+    int nkw[kMaxWaveLayers];    // column tiles per warp of each layer's CTAs (>= the register tiles)
+    int nkw_max;
+    unsigned stamp_base;        // the word of (layer, step s) carries stamp_base + s + 1
+    long long spin_limit;
+    int withhold_cta;
+    const uint4 *wfrag[kMaxWaveLayers];
+    const float *bias[kMaxWaveLayers];   // [H][4] (unit-major) bias of layers >= 1; layer 0's is in G
+    const float *G;             // [nsplit][T*B][H][4] layer 0's projection output incl. bias
+    long long g_split_stride;
+    const float *h0, *c0;       // [L][B][H] or nullptr
+    float *hT, *cT;             // [L][B][H] or nullptr
+    float *y;                   // [T][B][H]: the top layer's h
+    unsigned long long *xch;    // [L][T][B][H] exchange words, one slot per (layer, timestep)
+    int *status;
+};
+bool recur_wave_shape_ok(int mt, int nkr);
+size_t recur_wave_smem_bytes(int mt, int nkr, int nkw_max, int upc, int B);
+cudaError_t recur_wave_prepare(int mt, int nkr, int max_smem);
+cudaError_t launch_recur_wave(const RecurWaveArgs &a, int mt, int nkr, size_t smem, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------------
 // Register-resident sparse recurrent kernel (bf16 weights, CSR execution).  Same CTA/unit partition,
 // exchange buffer and finishing role as the dense register-resident kernel.  Warp w of a CTA owns the
 // columns [w * kspan, (w + 1) * kspan) of h; inside the warp every lane owns up to two of the CTA's 4 * units

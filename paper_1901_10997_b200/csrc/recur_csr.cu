@@ -119,14 +119,15 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArg
             } else if (!(probe & kProbeNoExchange)) {
                 const unsigned want = a.stamp_base + (unsigned)s;            // stamp of step s-1
                 const unsigned long long *src = xch_d + ((size_t)((s - 1) & 1) * B + b0) * H;
-                auto off = [&](int idx, int &so) -> bool {
+                auto off = [&](int idx, long long &so, unsigned &wnt) -> bool {
                     int b = 0, kk = idx;
                     if (!ONE) { b = idx / kspan; kk = idx - b * kspan; }
                     so = b * H + kbase + kk;
+                    wnt = want;
                     return kbase + kk < H;
                 };
                 auto sink = [&](int idx, float v) { hsw[idx] = v; };
-                poll_words<4>(src, nwords, lane, want, off, sink, abort_v, a.spin_limit, a.status);
+                poll_words<4>(src, nwords, lane, off, sink, abort_v, a.spin_limit, a.status);
             }
             __syncwarp();
 

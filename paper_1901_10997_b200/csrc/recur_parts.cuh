@@ -14,21 +14,22 @@
 namespace lstm {
 
 // Polls the words idx = lane, lane + 32, ... < nwords of one pass, KP per lane in flight per round trip.
-// off(idx, &word_offset) says where word idx lives relative to src and whether it exists; sink(idx, value)
-// receives every value once, as soon as its stamp equals `want`.
+// off(idx, &word_offset, &stamp) says where word idx lives relative to src, which stamp it must carry, and
+// whether it exists at all; sink(idx, value) receives every value once, as soon as its stamp is the wanted one.
 template <int KP, class OffFn, class Sink>
-__device__ __forceinline__ void poll_words(const unsigned long long *src, int nwords, int lane, unsigned want, OffFn off,
+__device__ __forceinline__ void poll_words(const unsigned long long *src, int nwords, int lane, OffFn off,
                                            Sink sink, volatile int *abort_v, long long spin_limit, int *status)
 {
     long long t_start = 0;
     for (int base = 0; base < nwords; base += 32 * KP) {
         unsigned pending = 0;
-        int soff[KP];
+        long long soff[KP];
+        unsigned want[KP];
 #pragma unroll
         for (int i = 0; i < KP; ++i) {
             const int idx = base + lane + 32 * i;
-            soff[i] = 0;
-            if (idx < nwords && off(idx, soff[i])) pending |= 1u << i;
+            soff[i] = 0; want[i] = 0;
+            if (idx < nwords && off(idx, soff[i], want[i])) pending |= 1u << i;
         }
         if (*abort_v) pending = 0;
         int rounds = 0;
@@ -39,7 +40,7 @@ __device__ __forceinline__ void poll_words(const unsigned long long *src, int nw
                 if (pending & (1u << i)) w[i] = ld_relaxed_u64(src + soff[i]);
 #pragma unroll
             for (int i = 0; i < KP; ++i)
-                if ((pending & (1u << i)) && (unsigned)(w[i] >> 32) == want) {
+                if ((pending & (1u << i)) && (unsigned)(w[i] >> 32) == want[i]) {
                     sink(base + lane + 32 * i, __uint_as_float((unsigned)w[i]));
                     pending &= ~(1u << i);
                 }
