@@ -102,6 +102,8 @@ typedef struct {
  *   LSTM_B200_RECUR = simt  shared-memory recurrent kernel instead of the register-resident one (bf16 dense or CSR)
  *                   = mma   no batched tensor-core recurrence (batches above four run as passes of four)
  *                   = tc1   batched tensor-core recurrence without cluster pairs
+ *   LSTM_B200_FUSE  = 0     never compute the input projection inside the recurrent kernel (single sequences of up
+ *                           to 40 steps on the register-resident kernel do so by default)
  *   LSTM_B200_WAVE  = 0     one launch per layer even where the layer-wavefront kernel would serve the stack
  *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
  *   LSTM_B200_COMPACT = 0   keep row/column-pruned units as explicit zeros, = 1 always run on the surviving units

@@ -32,6 +32,8 @@ struct Layer {
     int *wh_ptr[2] = {nullptr, nullptr};   // CSR recurrence: padded entry offsets [4H+1]
     void *wh_ent[2] = {nullptr, nullptr};
     uint4 *wfrag[2] = {nullptr, nullptr};  // register-resident kernel: operand-A fragments
+    uint4 *xfrag[2] = {nullptr, nullptr};  //   and Wx in the same layout (projection fused into the kernel's prologue)
+    int nkw_x = 0;
     __nv_bfloat16 *wtc = nullptr;          // batched tensor-core kernel: [D * ncta * RA][ld64] rows 4*unit+gate per CTA
     alignas(64) unsigned char tmap_wtc[128];
     uint4 *frag2[2] = {nullptr, nullptr};  // H-LSTM: fragments of the gate output matrices W
@@ -55,6 +57,7 @@ struct lstm_handle {
     // register-resident recurrent kernel (bf16 dense): row tiles, column tiles per warp in registers and
     // in shared memory, warps per CTA
     bool use_mma = false;
+    bool fuse_ok = false;              // short single sequences: projection fused into the register-resident kernel's prologue
     // register-resident sparse kernel (bf16, CSR execution): warps, columns per warp, row tiles, entry slots per lane
     bool use_csr_reg = false;
     int csr_nw = 0, csr_kspan = 0, csr_mt = 0, csr_slots = 0;
@@ -413,7 +416,7 @@ void free_all(lstm_handle *h)
 {
     for (auto &ly : h->layers) {
         cudaFree(ly.wx); cudaFree(ly.bias); cudaFree(ly.wx_rowptr); cudaFree(ly.wx_ent);
-        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); cudaFree(ly.frag2[d]); cudaFree(ly.csr_reg_ent[d]); cudaFree(ly.csr_reg_rows[d]); }
+        for (int d = 0; d < 2; ++d) { cudaFree(ly.wh[d]); cudaFree(ly.wh_ptr[d]); cudaFree(ly.wh_ent[d]); cudaFree(ly.wfrag[d]); cudaFree(ly.xfrag[d]); cudaFree(ly.frag2[d]); cudaFree(ly.csr_reg_ent[d]); cudaFree(ly.csr_reg_rows[d]); }
         cudaFree(ly.bias_out); cudaFree(ly.wtc);
     }
     cudaFree(h->G); cudaFree(h->xb0); cudaFree(h->xbn[0]); cudaFree(h->xbn[1]);
@@ -503,6 +506,11 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
     h->use_tc = want_tc(h);
     plan_mma(h);
     plan_wave(h);
+    {
+        const char *env = getenv("LSTM_B200_FUSE");
+        h->fuse_ok = h->use_mma && !(env && strcmp(env, "0") == 0) &&
+                     recur_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc, 1, false, true) <= (size_t)h->smem_optin - 64;
+    }
     if (csr && bf16) {
         // the register-resident sparse kernel: at most 16 units per CTA (warp w finishes unit w, a lane owns at
         // most two of the 4 * units rows); the entry slots per lane are known once every matrix has been laid out
@@ -588,6 +596,16 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                 if (rc) break;
                 std::vector<float> wave_x;
                 if (h->use_wave && l > 0) wave_x = m;                 // the wavefront kernel folds Wx of the upper layers into the step
+                if (h->use_mma && bf16 && h->fuse_ok) {
+                    // the same matrix as operand-A fragments: short single sequences compute their projection in the
+                    // recurrent kernel's prologue
+                    const int nranges = h->mma_nw / 2;                 // two warps share a column range
+                    ly.nkw_x = ((ly.in_l + 15) / 16 + nranges - 1) / nranges;
+                    const std::vector<uint32_t> fx = pack_fragments(m.data(), H, ly.in_l, h->ncta_dir, nranges, ly.nkw_x, h->mma_mt);
+                    rc = upload(h, (uint32_t **)&ly.xfrag[d], fx.data(), fx.size() * 4, st, "input weight fragments");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                    if (rc) break;
+                }
                 for (int q = 0; q < 4; ++q)
                     for (int j = 0; j < H; ++j) {
                         const float *srow = m.data() + (size_t)(q * H + j) * ly.in_l;
@@ -1222,8 +1240,10 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         const float *Xf = l == 0 ? x : h->ybuf[(l - 1) & 1];
         const int N = D * 4 * (h->Hh ? h->Hh : H);      // H-LSTM: the projection feeds the hidden layers
         int nsplit = 1;
-        // ---- input staging + projection
-        { const int prc = run_projection(h, l, l == 0 ? x : nullptr, Xf, M, N, &nsplit, st); if (prc != LSTM_OK) return prc; }
+        // ---- input staging + projection (a single short sequence on the register-resident kernel computes its
+        // projection inside that kernel's prologue instead: two launches and one round trip of G fewer per layer)
+        const bool fuse = h->fuse_ok && !h->Hh && B == 1 && T <= kFuseMaxT && !h->probe && ly.xfrag[0] != nullptr;
+        if (!fuse) { const int prc = run_projection(h, l, l == 0 ? x : nullptr, Xf, M, N, &nsplit, st); if (prc != LSTM_OK) return prc; }
 
         // ---- recurrence: all directions in one launch, or one launch per direction
         const int npass = h->seq_dirs ? D : 1;
@@ -1342,20 +1362,23 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.spin_limit = h->spin_limit;
             m.withhold_cta = h->withhold_cta;
             m.probe = B == 1 ? h->probe : 0;
-            for (int d = 0; d < D; ++d) m.wfrag[d] = ly.wfrag[d];
+            m.fuse = fuse ? 1 : 0;
+            m.in_l = ly.in_l; m.nkw_x = ly.nkw_x; m.X = Xf; m.bias = ly.bias;
+            m.gs_off = (int)recur_mma_fuse_gs_offset(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc);
+            for (int d = 0; d < D; ++d) { m.wfrag[d] = ly.wfrag[d]; m.xfrag[d] = ly.xfrag[d]; }
             m.G = h->G;
             m.g_split_stride = (long long)M * N;
             const size_t so = (size_t)l * D * B * H;
             m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
             m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
             m.y = l == L - 1 ? y : h->ybuf[l & 1];
-            m.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
+            m.xb_next = (l < L - 1 && h->use_tc && !fuse) ? h->xbn[l & 1] : nullptr;     // a fused next layer reads the fp32 activations
             m.xb_ld = h->ldn;
             m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
             m.xch = h->xch;
             m.status = h->status_dev;
             if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-            e = launch_recur_mma(m, h->mma_mt, h->mma_nkr, h->mma_nw, shp.smem, st);
+            e = launch_recur_mma(m, h->mma_mt, h->mma_nkr, h->mma_nw, fuse ? recur_mma_smem_bytes(h->mma_mt, h->mma_nkr, h->mma_nw, h->mma_nks, h->upc, 1, false, true) : shp.smem, st);
             ++h->last_launches;
             if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
             if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));

@@ -70,6 +70,13 @@ struct RecurMmaArgs {
     long long spin_limit;
     int withhold_cta;           // failure-path self-test: this CTA never publishes its h values (-1: none)
     int probe;                  // measurement only (kProbe* bits): parts of a step left out, outputs undefined
+    // fused input projection (one sequence of at most kFuseMaxT steps): the CTA computes its rows of G itself
+    int fuse;                   // 1: G is not read; X, xfrag, bias, in_l, nkw_x describe the projection
+    int in_l, nkw_x;            // input width; column tiles of Wx per column range (NW / 2 ranges, two warps each)
+    int gs_off;                 // byte offset of the finished rows of G in dynamic shared memory
+    const float *X;             // [T][in_l] this layer's input (fp32)
+    const uint4 *xfrag[2];      // Wx per direction in the fragment layout below with NW / 2 ranges of nkw_x tiles
+    const float *bias;          // [D][H][4]
     // per direction [cta][warp][column tile][row tile][lane] 16-byte operand-A fragments:
     // lane (g = lane / 4, p = lane % 4) holds rows g and g + 8, columns 2p, 2p+1 and 2p+8, 2p+9
     const uint4 *wfrag[2];
@@ -91,7 +98,9 @@ constexpr int kProbeNoExchange = 4;   // no wait for the other CTAs' words
 constexpr int kMmaTileCap16 = 18;   // MT * NKR limit with 16 warps (128 registers per thread, no spills)
 constexpr int kMmaTileCap8 = 40;    // ... with 8 warps
 bool recur_mma_shape_ok(int mt, int nkr, int nw);
-size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B, bool staged);
+size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B, bool staged, bool fused = false);
+size_t recur_mma_fuse_gs_offset(int mt, int nkr, int nw, int nkw_smem, int upc);
+constexpr int kFuseMaxT = 40;        // longest sequence whose projection the recurrent kernel computes in its prologue
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem);
 cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, size_t smem, cudaStream_t st);
 

@@ -29,6 +29,8 @@
 #include "common.cuh"
 #include "device_util.cuh"
 
+#include <algorithm>
+
 namespace lstm {
 namespace {
 
@@ -49,7 +51,10 @@ constexpr int kChunk = 4;     // batch rows per pass: hi and lo parts fill the 8
 // POLL3: a lane polls three words per round instead of four (single sequence, at most 96 columns per warp).
 // PROBE: the measurement build of the single-sequence variants, which honours a.probe (parts of a step left
 // out); in every other instantiation the probe tests fold away, so the production step carries none of them.
-template <int MT, int NKR, int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE = false>
+// FUSE: single short sequence (T <= kFuseMaxT): the CTA computes its own rows of the layer's input projection
+// G = X Wx^T + b in the prologue (Wx fragments streamed once from global memory, X split into bf16 hi + lo on
+// the fly) and keeps them in shared memory, instead of reading a G computed by a separate launch.
+template <int MT, int NKR, int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE = false, bool FUSE = false>
 __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArgs a)
 {
     const int probe = PROBE ? a.probe : 0;
@@ -77,9 +82,101 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
     uint4 *As = reinterpret_cast<uint4 *>(c_s + ((upc * B + 3) & ~3));            // [NW][nks][MT][32]
     // landing area of the exchange words of a pass over several batch rows: [NW][kChunk][kspan]
     unsigned long long *stage = reinterpret_cast<unsigned long long *>(As + (size_t)NW * nks * MT * 32);
+    // fused projection: this CTA's rows of G for every timestep, [kFuseMaxT][GP], behind everything else
+    constexpr int GP = MT * 16 + 1;
+    float *G_s = nullptr;
 
-    // ---- residency: this warp's tiles, registers first, the rest in shared memory
     const uint4 *wsrc = a.wfrag[d] + ((size_t)(cta * NW + warp) * nkw) * MT * 32 + lane;
+    if (FUSE) {
+        // ---- the CTA's rows of the input projection.  Both weight streams are requested into L2 at once, so that
+        // they leave HBM side by side; the registers the recurrent fragments will live in are free until the end.
+        // Work split: the NW / 2 column ranges of Wx are each taken by two warps, one for the first 24 timesteps
+        // and one for the rest, so that the accumulators of a warp stay few and two loads can be in flight.
+        constexpr int NR = NW / 2, NTH = 3;                       // column ranges; 8-step tiles per warp
+        const int range = warp >> 1, half = warp & 1;
+        const int nkx = a.nkw_x, in_l = a.in_l;
+        const uint4 *xbase = a.xfrag[d] + ((size_t)(cta * NR + range) * nkx) * MT * 32;
+        for (int i = lane + 32 * half; i < nkx * MT * 4; i += 64)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xbase) + (size_t)i * 128));
+        for (int i = lane; i < nkw * MT * 4; i += 32)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(wsrc - lane) + (size_t)i * 128));
+        float pacc[MT][NTH][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTH; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) pacc[mt][nt][e] = 0.0f;
+        const uint4 *xsrc = xbase + lane;
+        const int t0 = half * NTH * 8;
+        uint4 af[MT], an[MT];
+        float xv[NTH][4], xn[NTH][4];
+        auto fetch = [&](int i, uint4 (&fa)[MT], float (&fx)[NTH][4]) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) fa[mt] = i < nkx ? __ldg(xsrc + (size_t)(i * MT + mt) * 32) : make_uint4(0, 0, 0, 0);
+            const int k0 = (range * nkx + i) * 16 + 2 * tig;
+#pragma unroll
+            for (int nt = 0; nt < NTH; ++nt) {
+                const int t = t0 + nt * 8 + g;
+                const float *xr = a.X + (size_t)t * in_l;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int k = k0 + (e & 1) + (e >> 1) * 8;
+                    fx[nt][e] = (i < nkx && t < T && k < in_l) ? __ldg(xr + k) : 0.0f;
+                }
+            }
+        };
+        fetch(0, af, xv);
+#pragma unroll 1
+        for (int i = 0; i < nkx; ++i) {
+            fetch(i + 1, an, xn);
+#pragma unroll
+            for (int nt = 0; nt < NTH; ++nt) {
+                const __nv_bfloat162 h01 = __floats2bfloat162_rn(xv[nt][0], xv[nt][1]), h23 = __floats2bfloat162_rn(xv[nt][2], xv[nt][3]);
+                const __nv_bfloat162 l01 = __floats2bfloat162_rn(xv[nt][0] - __low2float(h01), xv[nt][1] - __high2float(h01));
+                const __nv_bfloat162 l23 = __floats2bfloat162_rn(xv[nt][2] - __low2float(h23), xv[nt][3] - __high2float(h23));
+                const unsigned bh0 = *reinterpret_cast<const unsigned *>(&h01), bh1 = *reinterpret_cast<const unsigned *>(&h23);
+                const unsigned bl0 = *reinterpret_cast<const unsigned *>(&l01), bl1 = *reinterpret_cast<const unsigned *>(&l23);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    mma_bf16(pacc[mt][nt], af[mt], bh0, bh1);
+                    mma_bf16(pacc[mt][nt], af[mt], bl0, bl1);
+                }
+            }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) af[mt] = an[mt];
+#pragma unroll
+            for (int nt = 0; nt < NTH; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) xv[nt][e] = xn[nt][e];
+        }
+        // every warp leaves its partial products in its own block (the blocks lie over shared memory that is only
+        // initialised afterwards); then each (timestep, row) adds its NR partial sums in a fixed order and the bias
+        constexpr int PP = MT * 16 + 1;
+        float *P = reinterpret_cast<float *>(smem) + (size_t)warp * (NTH * 8) * PP;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTH; ++nt) {
+                float *pp = P + (size_t)(nt * 8 + 2 * tig) * PP + mt * 16 + g;
+                pp[0] = pacc[mt][nt][0];
+                pp[PP] = pacc[mt][nt][1];
+                pp[8] = pacc[mt][nt][2];
+                pp[PP + 8] = pacc[mt][nt][3];
+            }
+        __syncthreads();
+        G_s = reinterpret_cast<float *>(smem + a.gs_off);
+        for (int i = tid; i < kFuseMaxT * MT * 16; i += NT) {
+            const int t = i / (MT * 16), r = i - t * (MT * 16);
+            const int hf = t / (NTH * 8), tl = t - hf * (NTH * 8);
+            float sum = r < 4 * nu ? a.bias[(size_t)d * 4 * H + (size_t)u0 * 4 + r] : 0.0f;
+#pragma unroll
+            for (int rg = 0; rg < NR; ++rg) sum += reinterpret_cast<const float *>(smem)[((size_t)(2 * rg + hf) * (NTH * 8) + tl) * PP + r];
+            G_s[(size_t)t * GP + r] = sum;
+        }
+        __syncthreads();
+    }
+    // ---- residency: this warp's tiles, registers first, the rest in shared memory
     uint4 areg[NKR][MT];
 #pragma unroll
     for (int i = 0; i < NKR; ++i)
@@ -129,7 +226,9 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 #pragma unroll
         for (int sp = 0; sp < kMaxSplit; ++sp) r.v[sp] = 0.0f;
         const int b = ci * kChunk + fb;
-        if (fin_warp && fpart == 0 && s < T && b < B) {
+        if (FUSE) {
+            if (fin_warp && fpart == 0 && s < T) r.v[0] = G_s[(size_t)(d ? (T - 1 - s) : s) * GP + warp * 4 + fq];
+        } else if (fin_warp && fpart == 0 && s < T && b < B) {
             const int t = d ? (T - 1 - s) : s;
             const float *gp = a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)(u0 + warp) * 4 + fq;
 #pragma unroll
@@ -359,36 +458,38 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
 
 typedef void (*KernelFn)(const RecurMmaArgs);
 
-template <int MT, int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE>
+template <int MT, int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE, bool FUSE>
 KernelFn pick_nkr(int nkr)
 {
     switch (nkr) {
-        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE, POLL3, PROBE>;
-        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE, POLL3, PROBE>;
-        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE, POLL3, PROBE>;
-        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE, (POLL3 && false), PROBE>;     // 128 columns per warp: four words
+        case 2: return recur_mma_kernel<MT, 2, NW, STAGED, ONE, POLL3, PROBE, FUSE>;
+        case 4: return recur_mma_kernel<MT, 4, NW, STAGED, ONE, POLL3, PROBE, FUSE>;
+        case 6: return recur_mma_kernel<MT, 6, NW, STAGED, ONE, POLL3, PROBE, FUSE>;
+        case 8: return recur_mma_kernel<MT, 8, NW, STAGED, ONE, (POLL3 && false), PROBE, FUSE>;     // 128 columns per warp: four words
         default: return nullptr;
     }
 }
-template <int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE = false>
+template <int NW, bool STAGED, bool ONE, bool POLL3, bool PROBE = false, bool FUSE = false>
 KernelFn pick_mt(int mt, int nkr)
 {
     switch (mt) {
-        case 1: return pick_nkr<1, NW, STAGED, ONE, POLL3, PROBE>(nkr);
-        case 2: return pick_nkr<2, NW, STAGED, ONE, POLL3, PROBE>(nkr);
-        case 3: return pick_nkr<3, NW, STAGED, ONE, POLL3, PROBE>(nkr);
-        case 4: return pick_nkr<4, NW, STAGED, ONE, POLL3, PROBE>(nkr);
+        case 1: return pick_nkr<1, NW, STAGED, ONE, POLL3, PROBE, FUSE>(nkr);
+        case 2: return pick_nkr<2, NW, STAGED, ONE, POLL3, PROBE, FUSE>(nkr);
+        case 3: return pick_nkr<3, NW, STAGED, ONE, POLL3, PROBE, FUSE>(nkr);
+        case 4: return pick_nkr<4, NW, STAGED, ONE, POLL3, PROBE, FUSE>(nkr);
         default: return nullptr;
     }
 }
 // variant 0: several rows polled from registers, 1: several rows staged in shared memory, 2: one sequence,
 // 3: one sequence with at most 96 columns per warp (three polled words per lane); 4, 5: the measurement
-// builds of 2 and 3
+// builds of 2 and 3; 6, 7: 2 and 3 with the input projection of a short sequence fused into the prologue
 KernelFn pick(int mt, int nkr, int nw, int variant)
 {
     if (!recur_mma_shape_ok(mt, nkr, nw)) return nullptr;
     if (variant == 4) return nw == 8 ? pick_mt<8, false, true, false, true>(mt, nkr) : pick_mt<16, false, true, false, true>(mt, nkr);
     if (variant == 5) return nw == 8 ? pick_mt<8, false, true, true, true>(mt, nkr) : pick_mt<16, false, true, true, true>(mt, nkr);
+    if (variant == 6) return nw == 8 ? pick_mt<8, false, true, false, false, true>(mt, nkr) : pick_mt<16, false, true, false, false, true>(mt, nkr);
+    if (variant == 7) return nw == 8 ? pick_mt<8, false, true, true, false, true>(mt, nkr) : pick_mt<16, false, true, true, false, true>(mt, nkr);
     if (variant == 1) return nw == 8 ? pick_mt<8, true, false, false>(mt, nkr) : pick_mt<16, true, false, false>(mt, nkr);
     if (variant == 2) return nw == 8 ? pick_mt<8, false, true, false>(mt, nkr) : pick_mt<16, false, true, false>(mt, nkr);
     if (variant == 3) return nw == 8 ? pick_mt<8, false, true, true>(mt, nkr) : pick_mt<16, false, true, true>(mt, nkr);
@@ -405,16 +506,26 @@ bool recur_mma_shape_ok(int mt, int nkr, int nw)
     return false;
 }
 
-size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B, bool staged)
+// fused projection: the partial products of all warps (24 timesteps x rows each) lie over the kernel's other
+// shared memory, the finished rows of G behind whichever is larger
+size_t recur_mma_fuse_gs_offset(int mt, int nkr, int nw, int nkw_smem, int upc)
+{
+    const size_t normal = recur_mma_smem_bytes(mt, nkr, nw, nkw_smem, upc, 1, false, false);
+    const size_t partial = (size_t)nw * 24 * (mt * 16 + 1) * 4;
+    return (std::max(normal, partial) + 15) & ~(size_t)15;
+}
+
+size_t recur_mma_smem_bytes(int mt, int nkr, int nw, int nkw_smem, int upc, int B, bool staged, bool fused)
 {
     const int nkw = nkr + nkw_smem;
-    return (staged ? (size_t)nw * kChunk * nkw * 16 * 8 : 0) + (size_t)nw * nkw * 256 + (size_t)2 * nw * (4 * (mt * 16 + 8) + 4) * 4 + (size_t)((upc * B + 3) & ~3) * 4 +
-           (size_t)nw * nkw_smem * mt * 512;
+    if (fused) return recur_mma_fuse_gs_offset(mt, nkr, nw, nkw_smem, upc) + (size_t)kFuseMaxT * (mt * 16 + 1) * 4;
+    return (staged ? (size_t)nw * kChunk * nkw * 16 * 8 : 0) + (size_t)nw * nkw * 256 + (size_t)2 * nw * (4 * (mt * 16 + 8) + 4) * 4 +
+           (size_t)((upc * B + 3) & ~3) * 4 + (size_t)nw * nkw_smem * mt * 512;
 }
 
 cudaError_t recur_mma_prepare(int mt, int nkr, int nw, int max_smem)
 {
-    for (int variant = 0; variant < 6; ++variant) {
+    for (int variant = 0; variant < 8; ++variant) {
         KernelFn fn = pick(mt, nkr, nw, variant);
         if (!fn) return cudaErrorInvalidValue;
         const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
@@ -427,8 +538,12 @@ cudaError_t launch_recur_mma(const RecurMmaArgs &a, int mt, int nkr, int nw, siz
 {
     int variant = a.staged ? 1 : a.B != 1 ? 0 : (nkr + a.nkw_smem) * 16 <= 96 ? 3 : 2;
     if (a.probe) {
-        if (variant < 2) return cudaErrorInvalidValue;      // probe modes exist for the single-sequence variants only
+        if (variant < 2 || a.fuse) return cudaErrorInvalidValue;      // probe modes exist for the plain single-sequence variants only
         variant += 2;
+    }
+    if (a.fuse) {
+        if (variant < 2 || a.T > kFuseMaxT || !a.xfrag[0] || !a.X) return cudaErrorInvalidValue;
+        variant += 4;
     }
     KernelFn fn = pick(mt, nkr, nw, variant);
     if (!fn) return cudaErrorInvalidValue;
