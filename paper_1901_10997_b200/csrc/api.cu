@@ -89,6 +89,7 @@ struct lstm_handle {
     cudaStream_t last_stream = nullptr;
     // host-buffer variant staging
     float *hx = nullptr, *hy = nullptr, *hh0 = nullptr, *hc0 = nullptr, *hhT = nullptr, *hcT = nullptr;
+    int *status_pinned = nullptr;      // pinned host word the host-buffer call copies the device status into
     // profiling
     bool prof = false;
     std::vector<cudaEvent_t> ev;
@@ -425,6 +426,7 @@ void free_all(lstm_handle *h)
     cudaFree(h->wave_xch);
     cudaFree(h->cmap); cudaFree(h->rem_idx); cudaFree(h->rem_bias);
     cudaFree(h->ch0); cudaFree(h->cc0); cudaFree(h->cy); cudaFree(h->chT); cudaFree(h->ccT);
+    if (h->status_pinned) cudaFreeHost(h->status_pinned);
     cudaFree(h->hx); cudaFree(h->hy); cudaFree(h->hh0); cudaFree(h->hc0); cudaFree(h->hhT); cudaFree(h->hcT);
     for (auto e : h->ev) cudaEventDestroy(e);
     cudaGetLastError();
@@ -1470,6 +1472,10 @@ int lstm_forward_host(lstm_handle *h, const float *x, int T, int B, const float 
         if (!rc) rc = dev_alloc(h, &h->hc0, smax * 4, false, st, "host-variant c0");
         if (!rc) rc = dev_alloc(h, &h->hhT, smax * 4, false, st, "host-variant hT");
         if (!rc) rc = dev_alloc(h, &h->hcT, smax * 4, false, st, "host-variant cT");
+        if (rc == LSTM_OK && cudaHostAlloc((void **)&h->status_pinned, sizeof(int), cudaHostAllocDefault) != cudaSuccess) {
+            cudaGetLastError();
+            rc = fail(h, LSTM_ERR_NOMEM, "pinned status word could not be allocated");
+        }
         if (rc) return rc;
     }
     const size_t xn = (size_t)T * B * h->in_dim, yn = (size_t)T * B * h->D * h->H, sn = (size_t)h->L * h->D * B * h->H;
@@ -1486,8 +1492,14 @@ int lstm_forward_host(lstm_handle *h, const float *x, int T, int B, const float 
     if (yn) e = cudaMemcpyAsync(y, h->hy, yn * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && hT && sn) e = cudaMemcpyAsync(hT, h->hhT, sn * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && cT && sn) e = cudaMemcpyAsync(cT, h->hcT, sn * 4, cudaMemcpyDeviceToHost, st);
+    // the device status of this very call travels with the results: one synchronisation, no blocking copy
+    int *status_dev = h->inner ? h->inner->status_dev : h->status_dev;
+    *h->status_pinned = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->status_pinned, status_dev, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(e));
-    return lstm_status(h);
+    if (*h->status_pinned != 0) return lstm_status(h);         // reads, reports and clears the recorded status
+    return LSTM_OK;
 }
 
 int lstm_destroy(lstm_handle *h)
