@@ -268,7 +268,7 @@ void unit_range_host(int H, int nc, int c, int &u0, int &n)
 }
 
 // Launch shape of the recurrent kernel for B batch rows.
-struct RecurShape { int BT; size_t smem; int w_smem_bytes; int units_res_min; bool staged = false; };
+struct RecurShape { int BT; size_t smem; int w_smem_bytes; int units_res_min; bool staged = false; bool stage_all = false; int threads = 0; };
 
 RecurShape recur_shape(const lstm_handle *h, int B, int layer)
 {
@@ -318,6 +318,17 @@ RecurShape recur_shape(const lstm_handle *h, int B, int layer)
     s.w_smem_bytes = (int)w;
     s.smem = f + w;
     s.units_res_min = 0;
+    s.threads = h->threads;
+    // several chunks of rows per step: when all B rows of h fit beside the whole slice, they are staged at once
+    // (one polling phase per step instead of one per chunk) and the (unit, chunk) pairs spread over the warps
+    const size_t f_all = (size_t)2 * round_up(B, pick) * h->Hs * 4 + c_bytes;      // whole chunks of rows per buffer
+    if (B > pick && f_all + need_w <= budget) {
+        s.stage_all = true;
+        s.smem = f_all + need_w;
+        s.w_smem_bytes = (int)need_w;
+        const int nchunk = (B + pick - 1) / pick;
+        s.threads = std::max(h->threads, std::min(512, 32 * h->upc * nchunk));
+    }
     return s;
 }
 
@@ -1390,7 +1401,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         memset(&a, 0, sizeof a);
         a.dir0 = h->seq_dirs ? pass : 0; a.ndirs = h->seq_dirs ? 1 : D;
         a.H = H; a.Hp8 = h->Hp8; a.Hs = h->Hs; a.B = B; a.T = T; a.D = D;
-        a.ncta_dir = h->ncta_dir; a.nsplit = nsplit; a.BT = shp.BT; a.w_smem_bytes = shp.w_smem_bytes;
+        a.ncta_dir = h->ncta_dir; a.nsplit = nsplit; a.BT = shp.BT; a.w_smem_bytes = shp.w_smem_bytes; a.stage_all = shp.stage_all ? 1 : 0;
         a.stamp_base = h->stamp_next;
         h->stamp_next += (unsigned)T + 1u;
         a.spin_limit = h->spin_limit;
@@ -1408,7 +1419,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         a.xch = h->xch;
         a.status = h->status_dev;
         if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
-        e = csr ? launch_recur_csr(a, bf16, h->threads, shp.smem, st) : launch_recur_dense(a, bf16, h->threads, shp.smem, st);
+        e = csr ? launch_recur_csr(a, bf16, shp.threads, shp.smem, st) : launch_recur_dense(a, bf16, shp.threads, shp.smem, st);
         ++h->last_launches;
         if (record(h, -1, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
         if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "recurrent launch failed (layer %d): %s", l, cudaGetErrorString(e));

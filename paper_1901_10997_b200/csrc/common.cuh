@@ -25,6 +25,7 @@ struct RecurArgs {
     int nsplit;         // partial planes of the projection output to add up
     int BT;             // batch rows processed per chunk (1, 2, 4 or 8)
     int w_smem_bytes;   // shared-memory bytes set aside for resident weights
+    int stage_all;      // 1: all B rows of h are staged at once (one polling phase per step), chunks of BT rows share them
     unsigned stamp_base;        // exchange words of step s carry stamp_base + s + 1
     long long spin_limit;       // clock64 ticks a wait may last before the kernel gives up
     int withhold_cta;           // failure-path self-test: this CTA never publishes its h values (-1: none)

@@ -185,8 +185,11 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
     const int upc = (H + a.ncta_dir - 1) / a.ncta_dir;
 
     // shared-memory carve-up: staged h (two buffers of BT rows), c state, resident weights
+    // (stage_all: two buffers of all B rows, so that a step polls its exchange words in one phase)
+    // (rounded up to whole chunks: the products of the last chunk read BT rows, the ones beyond B stay zero)
+    const int rows_staged = a.stage_all ? ((B + BT - 1) / BT) * BT : BT;
     float *h_s = reinterpret_cast<float *>(smem);
-    float *c_s = h_s + 2 * BT * Hs;
+    float *c_s = h_s + 2 * rows_staged * Hs;
     unsigned char *w_s = reinterpret_cast<unsigned char *>(c_s + ((upc * B + 3) & ~3));
 
     // ---- residency: how many leading units of this CTA live in shared memory
@@ -223,7 +226,7 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
     }
     const unsigned char *res_base = CSR ? w_s + ((4 * upc + 1 + 3) & ~3) * 4 : w_s;
 
-    for (int i = tid; i < 2 * BT * Hs; i += nthreads) h_s[i] = 0.0f;
+    for (int i = tid; i < 2 * rows_staged * Hs; i += nthreads) h_s[i] = 0.0f;
     for (int i = tid; i < nu * B; i += nthreads) {
         const int u = i / B, b = i - u * B;
         c_s[u * B + b] = a.c0 ? a.c0[((size_t)d * B + b) * H + u0 + u] : 0.0f;
@@ -238,9 +241,129 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
     const int b_mine = vidx % BT;           // its batch row inside the chunk
     const int b_gather = lane & (BT - 1);   // batch row a lane < BT finalises
 
+    // gates and state update of unit u for the batch rows b0 .. b0+nb-1 staged at hb; g_pl: the projection terms
+    // fetched ahead for this lane (valid when g_ahead), else they are loaded here
+    auto process_unit = [&](int u, int b0, int nb, const float *hb, bool g_ahead, const float (&g_pl)[4], int s, int t) {
+        AT acc[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] = (AT)0;
+        if (!CSR) {
+            // one copy of the loop serves resident (shared) and streamed (global) units: the
+            // base pointer is warp-uniform and the loads are generic
+            const WT *rows = (u < units_res) ? reinterpret_cast<const WT *>(res_base) + (size_t)u * 4 * a.Hp8
+                                             : wg + (size_t)u * 4 * a.Hp8;
+            unit_dot_dense<WT, BT, AT>(rows, a.Hp8, hb, Hs, lane, acc);
+        } else {
+            int e[5];
+#pragma unroll
+            for (int i = 0; i < 5; ++i) e[i] = rp_s[4 * u + i] - ent_base;
+            const ET *ents = (u < units_res) ? reinterpret_cast<const ET *>(res_base) : eg + ent_base;
+            unit_dot_csr<ET, BT, AT>(ents, e, hb, Hs, lane, acc);
+        }
+        AT z = warp_reduce_multi<V, AT>(acc, lane);
+
+        float g_in = (g_pl[0] + g_pl[1]) + (g_pl[2] + g_pl[3]);
+        if (!g_ahead) {
+            g_in = 0.0f;
+            if (b_mine < nb) {
+                const float *gp = a.G + (((size_t)t * B + b0 + b_mine) * D + d) * 4 * H +
+                                  (size_t)(u0 + u) * 4 + q_mine;
+                for (int sp = 0; sp < a.nsplit; ++sp)
+                    g_in += __ldg(gp + (size_t)sp * a.g_split_stride);
+            }
+        }
+        z += (AT)g_in;
+        const AT act = gate_fn(z, q_mine == 2);
+        const AT vi = __shfl_sync(0xffffffffu, act, (0 * BT + b_gather) << SH);
+        const AT vf = __shfl_sync(0xffffffffu, act, (1 * BT + b_gather) << SH);
+        const AT vg = __shfl_sync(0xffffffffu, act, (2 * BT + b_gather) << SH);
+        const AT vo = __shfl_sync(0xffffffffu, act, (3 * BT + b_gather) << SH);
+        if (lane < nb) {
+            const int b = b0 + lane;
+            const int j = u0 + u;
+            const AT cn_a = fma(vf, (AT)c_s[u * B + b], vi * vg);
+            const float cn = (float)cn_a;
+            const float hn = (float)(vo * tanh_t(cn_a));
+            if ((int)blockIdx.x != a.withhold_cta)
+            st_relaxed_u64(xch_d + ((size_t)(s & 1) * B + b) * H + j,
+                           ((unsigned long long)(a.stamp_base + (unsigned)s + 1u) << 32) |
+                               (unsigned long long)__float_as_uint(hn));
+            c_s[u * B + b] = cn;
+            a.y[((size_t)t * B + b) * D * H + (size_t)d * H + j] = hn;
+            if (a.xb_next) {
+                const size_t xi = ((size_t)t * B + b) * a.xb_ld + (size_t)d * H + j;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
+                a.xb_next[xi] = hi;
+                a.xb_next[a.xb_plane + xi] = __float2bfloat16_rn(hn - __bfloat162float(hi));
+            }
+            if (s == T - 1) {
+                if (a.hT) a.hT[((size_t)d * B + b) * H + j] = hn;
+                if (a.cT) a.cT[((size_t)d * B + b) * H + j] = cn;
+            }
+        }
+    };
+
 #pragma unroll 1
     for (int s = 0; s < T; ++s) {
         const int t = d ? (T - 1 - s) : s;
+        if (a.stage_all) {
+            // ---- all B rows of h_{t-1} in ONE polling phase (eight words per thread in flight over the flattened
+            // [B][H] block), then every (unit, chunk of BT rows) pair on its own warp
+            float *buf = h_s + (size_t)(s & 1) * rows_staged * Hs;
+            const int total = B * H;
+            if (s == 0) {
+                for (int i = tid; i < total; i += nthreads) {
+                    const int b = i / H, k = i - b * H;
+                    buf[b * Hs + h_pos<!CSR>(k, Hs)] = a.h0 ? a.h0[(size_t)d * B * H + i] : 0.0f;
+                }
+            } else {
+                const unsigned want = a.stamp_base + (unsigned)s;
+                const unsigned long long *src = xch_d + (size_t)((s - 1) & 1) * B * H;
+                long long t_start = 0;
+                bool gave_up = false;
+                for (int base = tid; base < total && !gave_up; base += 8 * nthreads) {
+                    unsigned pending = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) pending |= (base + i * nthreads < total) ? (1u << i) : 0u;
+                    int rounds = 0;
+                    while (pending) {
+                        unsigned long long w[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (pending & (1u << i)) w[i] = ld_relaxed_u64(src + base + i * nthreads);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if ((pending & (1u << i)) && (unsigned)(w[i] >> 32) == want) {
+                                const int idx = base + i * nthreads, b = idx / H, k = idx - b * H;
+                                buf[b * Hs + h_pos<!CSR>(k, Hs)] = __uint_as_float((unsigned)w[i]);
+                                pending &= ~(1u << i);
+                            }
+                        if (pending && ((++rounds & 63) == 0)) {
+                            const long long now = clock64();
+                            if (t_start == 0) t_start = now;
+                            if (now - t_start > a.spin_limit || ld_volatile_s32(a.status) != kStatusOk) {
+                                gave_up = true;
+                                break;
+                            }
+                        }
+                    }
+                }
+                if (gave_up) abort_s = 1;
+            }
+            __syncthreads();
+            if (abort_s) {
+                if (tid == 0) atomicExch(a.status, kStatusTimeout);
+                return;
+            }
+            const float no_g[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 1
+            for (int item = warp; item < nu * nchunk; item += nwarps) {
+                const int u = item / nchunk, ci = item - u * nchunk, b0 = ci * BT;
+                process_unit(u, b0, min(BT, B - b0), buf + (size_t)b0 * Hs, false, no_g, s, t);
+            }
+            __syncthreads();        // pacing, as below: polls only after this CTA's own stores
+            continue;
+        }
 #pragma unroll 1
         for (int ci = 0; ci < nchunk; ++ci) {
             const int b0 = ci * BT;
@@ -309,65 +432,7 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
 
             // ---- gates and state update, one unit per warp at a time
 #pragma unroll 1
-            for (int u = warp; u < nu; u += nwarps) {
-                AT acc[V];
-#pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = (AT)0;
-                if (!CSR) {
-                    // one copy of the loop serves resident (shared) and streamed (global) units: the
-                    // base pointer is warp-uniform and the loads are generic
-                    const WT *rows = (u < units_res) ? reinterpret_cast<const WT *>(res_base) + (size_t)u * 4 * a.Hp8
-                                                     : wg + (size_t)u * 4 * a.Hp8;
-                    unit_dot_dense<WT, BT, AT>(rows, a.Hp8, hb, Hs, lane, acc);
-                } else {
-                    int e[5];
-#pragma unroll
-                    for (int i = 0; i < 5; ++i) e[i] = rp_s[4 * u + i] - ent_base;
-                    const ET *ents = (u < units_res) ? reinterpret_cast<const ET *>(res_base) : eg + ent_base;
-                    unit_dot_csr<ET, BT, AT>(ents, e, hb, Hs, lane, acc);
-                }
-                AT z = warp_reduce_multi<V, AT>(acc, lane);
-
-                float g_in = (g_pl[0] + g_pl[1]) + (g_pl[2] + g_pl[3]);
-                if (u != warp) {
-                    g_in = 0.0f;
-                    if (b_mine < nb) {
-                        const float *gp = a.G + (((size_t)t * B + b0 + b_mine) * D + d) * 4 * H +
-                                          (size_t)(u0 + u) * 4 + q_mine;
-                        for (int sp = 0; sp < a.nsplit; ++sp)
-                            g_in += __ldg(gp + (size_t)sp * a.g_split_stride);
-                    }
-                }
-                z += (AT)g_in;
-                const AT act = gate_fn(z, q_mine == 2);
-                const AT vi = __shfl_sync(0xffffffffu, act, (0 * BT + b_gather) << SH);
-                const AT vf = __shfl_sync(0xffffffffu, act, (1 * BT + b_gather) << SH);
-                const AT vg = __shfl_sync(0xffffffffu, act, (2 * BT + b_gather) << SH);
-                const AT vo = __shfl_sync(0xffffffffu, act, (3 * BT + b_gather) << SH);
-                if (lane < nb) {
-                    const int b = b0 + lane;
-                    const int j = u0 + u;
-                    const AT cn_a = fma(vf, (AT)c_s[u * B + b], vi * vg);
-                    const float cn = (float)cn_a;
-                    const float hn = (float)(vo * tanh_t(cn_a));
-                    if ((int)blockIdx.x != a.withhold_cta)
-                    st_relaxed_u64(xch_d + ((size_t)(s & 1) * B + b) * H + j,
-                                   ((unsigned long long)(a.stamp_base + (unsigned)s + 1u) << 32) |
-                                       (unsigned long long)__float_as_uint(hn));
-                    c_s[u * B + b] = cn;
-                    a.y[((size_t)t * B + b) * D * H + (size_t)d * H + j] = hn;
-                    if (a.xb_next) {
-                        const size_t xi = ((size_t)t * B + b) * a.xb_ld + (size_t)d * H + j;
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
-                        a.xb_next[xi] = hi;
-                        a.xb_next[a.xb_plane + xi] = __float2bfloat16_rn(hn - __bfloat162float(hi));
-                    }
-                    if (s == T - 1) {
-                        if (a.hT) a.hT[((size_t)d * B + b) * H + j] = hn;
-                        if (a.cT) a.cT[((size_t)d * B + b) * H + j] = cn;
-                    }
-                }
-            }
+            for (int u = warp; u < nu; u += nwarps) process_unit(u, b0, nb, hb, u == warp, g_pl, s, t);
             // Pacing: no warp starts to poll for the next pass before this CTA has issued its own stores;
             // loads that spin on words that are not there yet would sit in front of those stores on the
             // way to L2 and delay every other CTA.
