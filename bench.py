@@ -427,16 +427,21 @@ class GpuCase:
         return float(np.mean([sum(int(np.count_nonzero(self.weights[l * w.dirs + d]["mask_h"])) for d in range(w.dirs))
                               for l in range(w.layers)]))
 
-    def roofline(self, rec_ms, rec_n, peak, peak_kind):
+    def roofline(self, rec_ms, rec_n, peak, peak_kind, fused=False):
         w = self.w
         alg_bytes = recurrence_bytes_per_launch(w, "hlstm" if self.mode == "hlstm" else self.nnz())
+        if fused:
+            # the launch also computes its layer's input projection: the input matrix and the activations once
+            wbytes = 2 if w.dtype == "bf16" else 4
+            in_avg = (w.in_dim + (w.layers - 1) * w.dirs * w.hidden) / w.layers
+            alg_bytes += w.dirs * 4.0 * w.hidden * in_avg * wbytes + w.T * w.B * in_avg * 4.0
         rec_avg_ms = rec_ms / max(rec_n, 1)
         achieved = alg_bytes / (rec_avg_ms * 1e-3) / 1e9 if rec_avg_ms > 0 else None
         info = self.model.info()
         kernel_name, kernel_src = kernel_of(info, self.mode)
         traffic, source = measured_traffic(kernel_name, self.name, kernel_src)
         steps_per_launch = w.T * (2 if (w.dirs == 2 and info.get("ctas_per_dir") == info.get("sm_count")) else 1)
-        return {"bound": "hbm", "kernel": f"{kernel_name} (one launch = one layer, all T steps)",
+        return {"bound": "hbm", "kernel": f"{kernel_name} (one launch = one layer, all T steps" + (", its input projection in the prologue)" if fused else ")"),
                 "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak if achieved else None), "peak_kind": f"of {peak_kind}",
                 "traffic": traffic, "traffic_source": source, "algorithmic_bytes_per_launch": alg_bytes,
@@ -447,14 +452,15 @@ class GpuCase:
     def on_chip(self, steps):
         """The yardstick that binds once the matrix is on-chip: the dependency chain of one step.  Uses the
         library's probe modes (parts of the step left out) on this very handle and workload; every figure is the
-        recurrent kernel's launch time / T, prologue included."""
+        recurrent kernel's launch time / T, prologue included, all from the measurement build of the kernel (projection as a
+        launch of its own, so that every mode has the same prologue)."""
         pkg, m, w = self.pkg, self.model, self.w
         try:
             m.probe(0)
         except pkg.LstmError:
             return None
         res = {}
-        modes = [("step_us", 0),
+        modes = [("step_us", pkg.LSTM_PROBE_WHOLE_STEP),
                  ("empty_step_us", pkg.LSTM_PROBE_NO_PRODUCTS | pkg.LSTM_PROBE_NO_GATES),
                  ("exchange_and_gates_us", pkg.LSTM_PROBE_NO_PRODUCTS),
                  ("compute_only_us", pkg.LSTM_PROBE_NO_EXCHANGE),
@@ -564,7 +570,7 @@ def run_gpu(args):
         ms_per_step = total_ms / args.steps
         seqs, us_per_seq, seqs_per_sec = job_throughput(world, w.B, ms_per_step)
         peak, peak_kind = measured_peaks()
-        roof = case.roofline(rec_ms, rec_n, peak, peak_kind)
+        roof = case.roofline(rec_ms, rec_n, peak, peak_kind, fused=(proj_ms == 0.0 and stage_ms == 0.0))
         gpu_launches = int(launches_per_fwd * args.steps)
         if world == 1 and not args.no_legs:
             oc = case.on_chip(min(args.steps, 20))
@@ -628,7 +634,7 @@ def run_legs(torch, pkg, dev, flush_buf, cache, peak, peak_kind):
                 "sequences_per_sec_p50": w.B / (p50 * 1e-3),
                 "gpu_launches": int(case.model.info()["launches_per_forward"] * steps),
                 "kernel_ms_per_forward": {"stage": stage_ms / nk, "projection": proj_ms / nk, "recurrence": rec_ms / nk},
-                "roofline": case.roofline(rec_ms, rec_n, peak, peak_kind),
+                "roofline": case.roofline(rec_ms, rec_n, peak, peak_kind, fused=(proj_ms == 0.0 and stage_ms == 0.0 and case.mode == "dense" and w.dtype == "bf16")),
                 "library": case.model.info(),
                 "clocks": clocks.summary(),
                 "wall_s": None,

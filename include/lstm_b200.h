@@ -219,11 +219,13 @@ LSTM_API int lstm_profile_read(lstm_handle *h, int *launches, float *ms);
  * leave parts of that chain out, so that timing them shows what each part costs (the "empty step": exchange
  * only, is the floor no kernel of this structure can go below).  Bits: LSTM_PROBE_NO_PRODUCTS (no tensor
  * instructions), LSTM_PROBE_NO_GATES (no reduction, gate functions or output stores; every unit still
- * publishes a word per step), LSTM_PROBE_NO_EXCHANGE (no waiting for other CTAs).  OUTPUTS ARE UNDEFINED
+ * publishes a word per step), LSTM_PROBE_NO_EXCHANGE (no waiting for other CTAs), LSTM_PROBE_WHOLE_STEP (nothing left
+ * out: the measurement build itself, with the projection as a launch of its own, as the yardstick the other modes
+ * are compared with; its outputs are valid).  With any other bit OUTPUTS ARE UNDEFINED
  * while a mask is set; 0 restores normal operation.  LSTM_ERR_UNSUPPORTED for handles that run another
  * recurrent kernel.  Every wait stays bounded in every mode.
  */
-enum { LSTM_PROBE_NO_PRODUCTS = 1, LSTM_PROBE_NO_GATES = 2, LSTM_PROBE_NO_EXCHANGE = 4 };
+enum { LSTM_PROBE_NO_PRODUCTS = 1, LSTM_PROBE_NO_GATES = 2, LSTM_PROBE_NO_EXCHANGE = 4, LSTM_PROBE_WHOLE_STEP = 8 };
 LSTM_API int lstm_probe(lstm_handle *h, int parts_left_out);
 
 /*

@@ -11,4 +11,4 @@ from .binding import (LSTM, HLSTM, LstmError, hlstm_create, lib_path, load_libra
                       LSTM_F32, LSTM_BF16W_F32S, LSTM_DENSE, LSTM_CSR, LSTM_OK, LSTM_ERR_INVALID,
                       LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT,
                       LSTM_K_STAGE, LSTM_K_PROJ, LSTM_K_RECUR, LSTM_K_COUNT,
-                      LSTM_PROBE_NO_PRODUCTS, LSTM_PROBE_NO_GATES, LSTM_PROBE_NO_EXCHANGE)
+                      LSTM_PROBE_NO_PRODUCTS, LSTM_PROBE_NO_GATES, LSTM_PROBE_NO_EXCHANGE, LSTM_PROBE_WHOLE_STEP)

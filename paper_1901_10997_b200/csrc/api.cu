@@ -1537,7 +1537,7 @@ int lstm_probe(lstm_handle *h, int parts_left_out)
 {
     if (!h) return LSTM_ERR_INVALID;
     if (h->inner) { const int rc = lstm_probe(h->inner, parts_left_out); if (rc) h->err = h->inner->err; return rc; }
-    if (parts_left_out < 0 || parts_left_out > 7) return fail(h, LSTM_ERR_INVALID, "probe mask %d outside 0..7", parts_left_out);
+    if (parts_left_out < 0 || parts_left_out > 15) return fail(h, LSTM_ERR_INVALID, "probe mask %d outside 0..15", parts_left_out);
     if (parts_left_out && ((!h->use_mma && !h->use_csr_reg) || h->Hh))
         return fail(h, LSTM_ERR_UNSUPPORTED, "only the register-resident recurrent kernels (dense and sparse) of an LSTM handle have probe modes");
     h->probe = parts_left_out;
