@@ -60,7 +60,10 @@ enum {
     LSTM_ERR_UNSUPPORTED = 2,  /* valid request the library cannot serve (e.g. hidden >= 65536)            */
     LSTM_ERR_CUDA = 3,         /* a CUDA call failed (no device, launch refused ...)                        */
     LSTM_ERR_NOMEM = 4,        /* host or device allocation failed                                           */
-    LSTM_ERR_TIMEOUT = 5       /* a device-side wait of the recurrent kernel gave up; outputs undefined     */
+    LSTM_ERR_TIMEOUT = 5,      /* a device-side wait of the recurrent kernel gave up; outputs undefined     */
+    LSTM_ERR_INTERNAL = 6      /* checked build only (liblstm_b200_checked.so, compiled with -DLSTM_B200_CHECKED):
+                                  an index or shared-memory carve-up check inside a kernel failed; the access
+                                  was skipped, nothing trapped; outputs undefined                            */
 };
 
 /* how the recurrent and input matrices are executed */

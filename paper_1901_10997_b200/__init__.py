@@ -9,6 +9,6 @@ from .binding import (LSTM, HLSTM, LstmError, hlstm_create, lib_path, load_libra
                       lstm_probe, lstm_profile_enable, lstm_profile_read, lstm_selftest_timeout, lstm_status,
                       lstm_lhp_points, lstm_nearest_lhp, lstm_fold_input_affine, lstm_csr_lane_layout,
                       LSTM_F32, LSTM_BF16W_F32S, LSTM_DENSE, LSTM_CSR, LSTM_OK, LSTM_ERR_INVALID,
-                      LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT,
+                      LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT, LSTM_ERR_INTERNAL,
                       LSTM_K_STAGE, LSTM_K_PROJ, LSTM_K_RECUR, LSTM_K_COUNT,
                       LSTM_PROBE_NO_PRODUCTS, LSTM_PROBE_NO_GATES, LSTM_PROBE_NO_EXCHANGE, LSTM_PROBE_WHOLE_STEP)

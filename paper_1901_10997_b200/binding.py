@@ -13,11 +13,15 @@ import numpy as np
 
 LSTM_F32, LSTM_BF16W_F32S = 0, 1
 LSTM_DENSE, LSTM_CSR = 0, 1
-LSTM_OK, LSTM_ERR_INVALID, LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT = range(6)
+LSTM_OK, LSTM_ERR_INVALID, LSTM_ERR_UNSUPPORTED, LSTM_ERR_CUDA, LSTM_ERR_NOMEM, LSTM_ERR_TIMEOUT, LSTM_ERR_INTERNAL = range(7)
 LSTM_K_STAGE, LSTM_K_PROJ, LSTM_K_RECUR, LSTM_K_COUNT = 0, 1, 2, 3
 LSTM_PROBE_NO_PRODUCTS, LSTM_PROBE_NO_GATES, LSTM_PROBE_NO_EXCHANGE, LSTM_PROBE_WHOLE_STEP = 1, 2, 4, 8
 
-_LIB_PATH = Path(__file__).resolve().parent / "liblstm_b200.so"
+import os as _os
+
+# LSTM_B200_LIBRARY=checked loads the build with index checks compiled into the kernels (same ABI)
+_LIB_PATH = Path(__file__).resolve().parent / ("liblstm_b200_checked.so" if _os.environ.get("LSTM_B200_LIBRARY") == "checked"
+                                               else "liblstm_b200.so")
 _lib = None
 
 

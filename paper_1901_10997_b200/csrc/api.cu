@@ -1461,7 +1461,9 @@ int lstm_status(lstm_handle *h)
     if (e != cudaSuccess) return fail(h, LSTM_ERR_CUDA, "status read failed: %s", cudaGetErrorString(e));
     if (v != 0) {
         cudaMemset(status_dev, 0, sizeof v);
-        return fail(h, v, v == LSTM_ERR_TIMEOUT ? "a device-side wait gave up (timeout); outputs are undefined" : "device reported status %d", v);
+        return fail(h, v, v == LSTM_ERR_TIMEOUT ? "a device-side wait gave up (timeout); outputs are undefined"
+                          : v == LSTM_ERR_INTERNAL ? "an index check of the checked build failed inside a kernel; outputs are undefined"
+                                                   : "device reported status %d", v);
     }
     return LSTM_OK;
 }

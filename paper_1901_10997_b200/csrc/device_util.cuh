@@ -11,6 +11,35 @@
 namespace lstm {
 
 // ---------------------------------------------------------------------------------------------------
+// Checked build (-DLSTM_B200_CHECKED): the stand-in for a memory checker.  Index and carve-up checks compile
+// into the kernels; a violation records kStatusInternal in the status word (reported as LSTM_ERR_INTERNAL) and
+// the access is skipped -- nothing traps, nothing reads or writes out of range.  In the normal build the macros
+// vanish.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kStatusInternal = 6;
+__device__ __forceinline__ unsigned dynamic_smem_bytes()
+{
+    unsigned v;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(v));
+    return v;
+}
+#ifdef LSTM_B200_CHECKED
+__device__ __forceinline__ bool check_index(long long i, long long n, int *status)
+{
+    if (i >= 0 && i < n) return true;
+    atomicCAS(status, 0, kStatusInternal);
+    return false;
+}
+#define LSTM_CHECK_INDEX(i, n, status) lstm::check_index((long long)(i), (long long)(n), (status))
+// end_bytes: bytes of dynamic shared memory the kernel is about to carve up (or read as an operand)
+#define LSTM_CHECK_SMEM_END(end_bytes, status) \
+    do { if ((unsigned long long)(end_bytes) > (unsigned long long)lstm::dynamic_smem_bytes()) atomicCAS((status), 0, lstm::kStatusInternal); } while (0)
+#else
+#define LSTM_CHECK_INDEX(i, n, status) true
+#define LSTM_CHECK_SMEM_END(end_bytes, status) do { } while (0)
+#endif
+
+// ---------------------------------------------------------------------------------------------------
 // global-memory accesses of the exchange
 // ---------------------------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)

@@ -191,6 +191,7 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
     float *h_s = reinterpret_cast<float *>(smem);
     float *c_s = h_s + 2 * rows_staged * Hs;
     unsigned char *w_s = reinterpret_cast<unsigned char *>(c_s + ((upc * B + 3) & ~3));
+    LSTM_CHECK_SMEM_END((size_t)(w_s - smem) + (size_t)a.w_smem_bytes, a.status);
 
     // ---- residency: how many leading units of this CTA live in shared memory
     int units_res = 0;

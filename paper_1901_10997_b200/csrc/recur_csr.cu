@@ -55,6 +55,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArg
     float *hs = reinterpret_cast<float *>(smem);                 // [NW][hstride]: NB rows of kspan staged h values
     float *red = hs + (size_t)NW * hstride;                      // [2][NW][WS]
     float *c_s = red + 2 * NW * WS;                              // [upc][B]
+    LSTM_CHECK_SMEM_END((size_t)(reinterpret_cast<unsigned char *>(c_s + ((upc * B + 3) & ~3)) - smem), a.status);
 
     // ---- residency: this lane's entry list and its rows
     unsigned ent[E];
@@ -144,6 +145,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArg
                     const float v = __uint_as_float(w & 0xffff0000u);
                     const unsigned off = hsw_off | (w & 0x7ffcu);
                     const bool second = (w & 0x8000u) != 0;
+                    if (!LSTM_CHECK_INDEX((w & 0x7ffcu) + (unsigned)((NB - 1) * kspan) * 4u, (unsigned)hstride * 4u, a.status)) continue;
 #pragma unroll
                     for (int b = 0; b < NB; ++b) {
                         const float hv = *reinterpret_cast<const float *>(smem + off + (unsigned)(b * kspan) * 4u);

@@ -85,6 +85,9 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
     // fused projection: this CTA's rows of G for every timestep, [kFuseMaxT][GP], behind everything else
     constexpr int GP = MT * 16 + 1;
     float *G_s = nullptr;
+    LSTM_CHECK_SMEM_END(reinterpret_cast<unsigned char *>(stage) - smem + (STAGED ? (size_t)NW * kChunk * kspan * 8 : 0), a.status);
+    if (FUSE) LSTM_CHECK_SMEM_END((size_t)a.gs_off + (size_t)kFuseMaxT * GP * 4, a.status);
+    if (FUSE) LSTM_CHECK_SMEM_END((size_t)NW * 24 * GP * 4, a.status);
 
     const uint4 *wsrc = a.wfrag[d] + ((size_t)(cta * NW + warp) * nkw) * MT * 32 + lane;
     if (FUSE) {
@@ -354,8 +357,10 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
                             if ((pending & (1u << i)) && (unsigned)(w[i] >> 32) == want) {
                                 const float v = __uint_as_float((unsigned)w[i]);
                                 const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-                                Bw[doff[i]] = hi;
-                                Bw[doff[i] + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
+                                if (LSTM_CHECK_INDEX(doff[i] + 16, nkw * 128, a.status)) {
+                                    Bw[doff[i]] = hi;
+                                    Bw[doff[i] + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
+                                }
                                 pending &= ~(1u << i);
                             }
                         if (pending && ((++rounds & 63) == 0)) {
@@ -396,10 +401,12 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_mma_kernel(const RecurMmaArg
             }
             // accumulator columns 2*tig and 2*tig+1 are the hi and lo parts of batch row tig
             float *rw = red + (size_t)((it & 1) * NW + warp) * WS + tig * RP + g;
+            if (LSTM_CHECK_INDEX((rw - red) + (MT - 1) * 16 + 8, 2 * NW * WS, a.status)) {
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                rw[mt * 16] = acc[mt][0] + acc[mt][1];
-                rw[mt * 16 + 8] = acc[mt][2] + acc[mt][3];
+                for (int mt = 0; mt < MT; ++mt) {
+                    rw[mt * 16] = acc[mt][0] + acc[mt][1];
+                    rw[mt * 16 + 8] = acc[mt][2] + acc[mt][3];
+                }
             }
 
             // ---- all partial sums of this pass are in place (two barriers and two buffers alternate)

@@ -136,6 +136,9 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     const int zld = 4 * upc;
     float *c_s = zs + zld * B;                                              // [B][units of this CTA]
     float *zs2 = c_s + ((upc * B + 3) & ~3);                                // [B][4*upc] the partner's partial sums (pair mode)
+    // checked build: the carve-up ends inside the launch's shared memory, and so does the 128-row read of the last weight tile
+    LSTM_CHECK_SMEM_END((size_t)(reinterpret_cast<unsigned char *>(zs2 + (pair ? zld * B : 0)) - smem_raw), a.status);
+    LSTM_CHECK_SMEM_END((size_t)(a_tiles - smem_u32(smem_raw)) + (size_t)(nkb_alloc - 1) * RT * 128 + (size_t)128 * 128, a.status);
 
     if (tid == 0) {
         abort_s = 0;

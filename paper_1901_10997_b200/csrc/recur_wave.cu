@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_wave_kernel(const RecurWaveA
     float *red = reinterpret_cast<float *>(smem + (size_t)NW * nkw_max * 256);    // [2][NW][WS]
     float *c_s = red + 2 * NW * WS;                                               // [upc][B]
     uint4 *As = reinterpret_cast<uint4 *>(c_s + ((upc * B + 3) & ~3));            // [NW][nks][MT][32]
+    LSTM_CHECK_SMEM_END((size_t)(reinterpret_cast<unsigned char *>(As + (size_t)NW * (nkw_max - NKR) * MT * 32) - smem), a.status);
 
     // ---- residency: this warp's tiles, registers first, the rest in shared memory
     const uint4 *wsrc = a.wfrag[layer] + ((size_t)(cta * NW + warp) * nkw) * MT * 32 + lane;
@@ -116,6 +117,7 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_wave_kernel(const RecurWaveA
             if (!ONE) { b = idx / kspan; kk = idx - b * kspan; }
             const int dof = ((kk >> 4) * 8 + 2 * b) * 16 + (kk & 15);
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            if (!LSTM_CHECK_INDEX(dof + 16, nkw * 128, a.status)) return;
             Bw[dof] = hi;
             Bw[dof + 16] = __float2bfloat16_rn(v - __bfloat162float(hi));
         };

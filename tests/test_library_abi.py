@@ -57,3 +57,11 @@ def test_create_rejects_bad_arguments_before_touching_the_device():
     assert "bad argument" in pkg.lstm_last_error(None)
     rc, _ = pkg.lstm_create(1, 3, 70000, 0, pkg.LSTM_F32, 1, pkg.LSTM_DENSE, 1, 1)
     assert rc == pkg.LSTM_ERR_UNSUPPORTED
+
+
+def test_checked_build_exports_the_same_boundary():
+    """liblstm_b200_checked.so (index checks compiled into the kernels) has the ABI of the normal build."""
+    from paper_1901_10997_b200 import build
+    lib = ctypes.CDLL(str(build.build(checked=True)))
+    for name in declared_functions():
+        assert hasattr(lib, name), name
