@@ -327,7 +327,8 @@ RecurShape recur_shape(const lstm_handle *h, int B, int layer)
         s.smem = f_all + need_w;
         s.w_smem_bytes = (int)need_w;
         const int nchunk = (B + pick - 1) / pick;
-        s.threads = std::max(h->threads, std::min(512, 32 * h->upc * nchunk));
+        (void)nchunk;
+        s.threads = 512;                 // all hands for the one polling phase: B * H words, eight per thread in flight
     }
     return s;
 }
@@ -1221,7 +1222,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         h->stamp_next = 1;
     }
 
-    if (h->use_wave && B <= 4) {
+    if (h->use_wave && B <= 4 && !h->probe) {          // (the probe builds exist for the per-layer kernels)
         // all layers in one launch: layer 0's projection for all timesteps, then the wavefront kernel
         int nsplit = 1;
         { const int prc = run_projection(h, 0, x, x, M, D * 4 * H, &nsplit, st); if (prc != LSTM_OK) return prc; }

@@ -312,6 +312,17 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
             // [B][H] block), then every (unit, chunk of BT rows) pair on its own warp
             float *buf = h_s + (size_t)(s & 1) * rows_staged * Hs;
             const int total = B * H;
+            // projection terms of this warp's first (unit, chunk) item, requested before the wait
+            float g_first[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            if (warp < nu * nchunk) {
+                const int u = warp / nchunk, b0 = (warp - u * nchunk) * BT;
+                if (b0 + b_mine < B) {
+                    const float *gp = a.G + (((size_t)t * B + b0 + b_mine) * D + d) * 4 * H + (size_t)(u0 + u) * 4 + q_mine;
+#pragma unroll
+                    for (int sp = 0; sp < 4; ++sp)
+                        if (sp < a.nsplit) g_first[sp] = ld_nc_early(gp + (size_t)sp * a.g_split_stride);
+                }
+            }
             if (s == 0) {
                 for (int i = tid; i < total; i += nthreads) {
                     const int b = i / H, k = i - b * H;
@@ -360,7 +371,8 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
 #pragma unroll 1
             for (int item = warp; item < nu * nchunk; item += nwarps) {
                 const int u = item / nchunk, ci = item - u * nchunk, b0 = ci * BT;
-                process_unit(u, b0, min(BT, B - b0), buf + (size_t)b0 * Hs, false, no_g, s, t);
+                if (item == warp) process_unit(u, b0, min(BT, B - b0), buf + (size_t)b0 * Hs, true, g_first, s, t);
+                else process_unit(u, b0, min(BT, B - b0), buf + (size_t)b0 * Hs, false, no_g, s, t);
             }
             __syncthreads();        // pacing, as below: polls only after this CTA's own stores
             continue;

@@ -391,3 +391,46 @@ def test_random_batched_shapes(oracle, c):
     ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
     got = run_gpu(w, weights, x, h0, c0)
     assert_close(got, ref, "bf16", "fuzz batched")
+
+
+# ---------------------------------------------------------------- the step-cost probe
+def test_probe_modes_run_to_the_end_and_the_whole_step_mode_is_exact(oracle):
+    """lstm_probe selects measurement builds that leave parts of the recurrent step out.  Every mode must run to
+    its end without a timeout (the exchange still completes: every unit publishes a word per step), the whole-step
+    mode must give the normal results, and handles on other kernels must refuse a mask."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    for mode, density in (("dense", 1.0), ("csr", 0.2)):
+        w = small("probe", 2, False, 48, 300, 9, 1, "bf16", density=density, seed=55)
+        weights, x = wl.make(w)
+        ref = oracle.forward(weights, x, layers=2, bidir=False, hidden=300)
+        m = pkg.LSTM(weights, layers=2, in_dim=48, hidden=300, dtype="bf16", exec_mode=mode, max_T=w.T, max_B=1)
+        xd = torch.from_numpy(x).cuda()
+        for mask in (pkg.LSTM_PROBE_NO_PRODUCTS, pkg.LSTM_PROBE_NO_GATES, pkg.LSTM_PROBE_NO_EXCHANGE,
+                     pkg.LSTM_PROBE_NO_PRODUCTS | pkg.LSTM_PROBE_NO_GATES, pkg.LSTM_PROBE_NO_EXCHANGE | pkg.LSTM_PROBE_NO_GATES):
+            if mode == "csr" and m.info()["layer_wavefront"]:
+                break
+            try:
+                m.probe(mask)
+            except pkg.LstmError as e:                     # a stack served by the wavefront kernel has no probe build
+                assert e.code == pkg.LSTM_ERR_UNSUPPORTED
+                break
+            m.forward(xd)
+            assert m.status() == pkg.LSTM_OK, (mode, mask)
+        if m.info()["recur_register_resident"] or m.info()["recur_csr_register_resident"]:
+            m.probe(pkg.LSTM_PROBE_WHOLE_STEP)
+            y, hT, cT = m.forward(xd)
+            m.check()
+            assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"probe whole step {mode}")
+        m.probe(0)
+        y, hT, cT = m.forward(xd)
+        m.check()
+        assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"after the probe {mode}")
+        m.close()
+    wf = small("probe_fp32", 1, False, 8, 20, 3, 1, "fp32", seed=56)
+    weights, x = wl.make(wf)
+    m = pkg.LSTM(weights, layers=1, in_dim=8, hidden=20, dtype="fp32", max_T=3, max_B=1)
+    with pytest.raises(pkg.LstmError) as e:
+        m.probe(pkg.LSTM_PROBE_NO_PRODUCTS)
+    assert e.value.code == pkg.LSTM_ERR_UNSUPPORTED
+    m.close()
