@@ -326,6 +326,9 @@ LSTM_API int lstm_csr_lane_layout(const int32_t *rowptr, const int32_t *col, con
  * enqueues on cuda_stream and synchronises that stream before returning, so a device-side timeout of
  * this very call is returned as LSTM_ERR_TIMEOUT.
  * err (may be NULL): caller-owned buffer of errlen bytes that receives the reason of a failure.
+ * Failure-path self-test: with LSTM_B200_NOALLOC_SELFTEST=<cta>:<clock ticks> in the environment, that CTA withholds
+ * its exchange words, the other CTAs' bounded waits run out after the given ticks, and the call returns
+ * LSTM_ERR_TIMEOUT with the CUDA context intact (nothing faults or hangs); the next call without it is normal again.
  */
 #define LSTM_NOALLOC_MAX_BH 8192
 LSTM_API int lstm_forward_noalloc(const float *wx, const float *wh, const float *b, int in_dim, int hidden,

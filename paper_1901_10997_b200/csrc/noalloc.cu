@@ -16,6 +16,7 @@
 #include <cuda_runtime.h>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 namespace {
@@ -38,6 +39,8 @@ struct Args {
     const float *wx, *wh, *b, *x, *h0, *c0;
     float *y, *hT, *cT;
     int in_dim, H, T, B, ncta;
+    int withhold_cta;           // failure-path self-test: this CTA never publishes its words (-1: none)
+    long long spin_limit;       // clock64 ticks a wait may last
     Scratch *scratch;
 };
 
@@ -96,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 1) recur_noalloc_kernel(const Args a
                     if ((++rounds & 63) == 0) {
                         const long long now = clock64();
                         if (t_start == 0) t_start = now;
-                        if (now - t_start > kSpinLimit || *(volatile int *)&sc->status != 0) { abort_s = 1; break; }
+                        if (now - t_start > a.spin_limit || *(volatile int *)&sc->status != 0) { abort_s = 1; break; }
                     }
                     w = ld_relaxed_u64(src + i);
                 }
@@ -143,6 +146,7 @@ __global__ void __launch_bounds__(kThreads, 1) recur_noalloc_kernel(const Args a
                 const float cn = (float)cn_d;
                 const float hn = (float)(go * tanh(cn_d));
                 c_s[u * B + bb] = cn;
+                if ((int)blockIdx.x != a.withhold_cta)
                 st_relaxed_u64(&sc->xch[s & 1][(size_t)bb * H + j],
                                ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned long long)__float_as_uint(hn));
                 a.y[((size_t)s * B + bb) * H + j] = hn;
@@ -243,6 +247,14 @@ extern "C" int lstm_forward_noalloc(const float *wx, const float *wh, const floa
     a.in_dim = in_dim; a.H = hidden; a.T = T; a.B = B;
     a.ncta = hidden < ds.sm_count ? hidden : ds.sm_count;
     a.scratch = ds.scratch;
+    a.withhold_cta = -1;
+    a.spin_limit = kSpinLimit;
+    // Failure-path self-test (see the header): LSTM_B200_NOALLOC_SELFTEST=<cta>:<clock ticks> makes that CTA withhold its
+    // words, so the other CTAs' waits run out after the given ticks and the call returns LSTM_ERR_TIMEOUT.
+    if (const char *env = getenv("LSTM_B200_NOALLOC_SELFTEST")) {
+        int cta = -1; long long ticks = 0;
+        if (sscanf(env, "%d:%lld", &cta, &ticks) == 2 && cta >= 0 && cta < a.ncta && ticks > 0) { a.withhold_cta = cta; a.spin_limit = ticks; }
+    }
     const int upc = (hidden + a.ncta - 1) / a.ncta;
     const size_t smem = ((size_t)B * (in_dim + hidden) + (size_t)upc * B) * sizeof(float);
     if (smem > (size_t)ds.smem_optin - 1024)

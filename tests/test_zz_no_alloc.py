@@ -71,3 +71,27 @@ def test_sizes_beyond_the_built_in_scratch_are_rejected():
     assert rc == pkg.LSTM_ERR_UNSUPPORTED and "scratch" in msg
     rc, msg = pkg.lstm_forward_noalloc(p, p, p, 0, 4, p, 2, 2, 0, 0, p, 0, 0)
     assert rc == pkg.LSTM_ERR_INVALID
+
+
+def test_withheld_words_end_in_a_timeout_not_a_hang(oracle, monkeypatch):
+    """One CTA withholds its exchange words: the bounded waits of the others run out after a millisecond, the call
+    returns LSTM_ERR_TIMEOUT, and the next call (the scratch array is cleared on entry) computes correctly."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    w = wl.Workload("noalloc_timeout", 1, False, 20, 70, 5, 2, "fp32", 0.3, seed=33)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    dev = torch.device("cuda:0")
+    t = {k: torch.from_numpy(np.ascontiguousarray(weights[0][k])).to(dev) for k in ("wx", "wh", "b")}
+    xd, hd, cd = (torch.from_numpy(a).to(dev) for a in (x, h0[0], c0[0]))
+    y = torch.zeros((w.T, w.B, w.hidden), device=dev)
+    args = (t["wx"].data_ptr(), t["wh"].data_ptr(), t["b"].data_ptr(), w.in_dim, w.hidden, xd.data_ptr(), w.T, w.B,
+            hd.data_ptr(), cd.data_ptr(), y.data_ptr(), 0, 0, torch.cuda.current_stream().cuda_stream)
+    monkeypatch.setenv("LSTM_B200_NOALLOC_SELFTEST", "3:2000000")
+    rc, msg = pkg.lstm_forward_noalloc(*args)
+    assert rc == pkg.LSTM_ERR_TIMEOUT and "timeout" in msg
+    monkeypatch.delenv("LSTM_B200_NOALLOC_SELFTEST")
+    ref = oracle.forward(weights, x, h0, c0, layers=1, bidir=False, hidden=w.hidden)
+    got = _noalloc_path(pkg, torch, w, weights, x, h0, c0)
+    floored, scaled = wl.rel_err(got[0], ref[0])
+    assert floored <= wl.TOLERANCE["fp32"], (floored, scaled)
