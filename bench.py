@@ -460,7 +460,7 @@ class GpuCase:
         except pkg.LstmError:
             return None
         res = {}
-        modes = [("step_us", pkg.LSTM_PROBE_WHOLE_STEP),
+        modes = [("step_us_probe_build", pkg.LSTM_PROBE_WHOLE_STEP),
                  ("empty_step_us", pkg.LSTM_PROBE_NO_PRODUCTS | pkg.LSTM_PROBE_NO_GATES),
                  ("exchange_and_gates_us", pkg.LSTM_PROBE_NO_PRODUCTS),
                  ("compute_only_us", pkg.LSTM_PROBE_NO_EXCHANGE),
@@ -475,8 +475,32 @@ class GpuCase:
             m.probe(0)
         self.step()                 # leave valid outputs behind
         m.check()
+        # The production step, from the production instantiation of the same kernel with the projection as a launch
+        # of its own (same prologue as the probe modes): a second handle on the same weights with the fused prologue
+        # switched off.  The probe builds carry run-time tests in the step (about 12 % on the whole step), so
+        # step_us_probe_build is above step_us; the modes that leave parts out are what they are for.
+        old = os.environ.get("LSTM_B200_FUSE")
+        os.environ["LSTM_B200_FUSE"] = "0"
+        try:
+            plain = pkg.LSTM(self.weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
+                             exec_mode=self.mode, max_T=w.T, max_B=w.B)
+        finally:
+            if old is None:
+                os.environ.pop("LSTM_B200_FUSE", None)
+            else:
+                os.environ["LSTM_B200_FUSE"] = old
+        keep = self.model
+        self.model = plain
+        try:
+            rec_ms, rec_n, _p, _s = self.kernel_split(steps)
+            plain.check()
+        finally:
+            self.model = keep
+            plain.close()
+        res["step_us"] = rec_ms / max(rec_n, 1) * 1e3 / w.T
         res["step_over_empty_step"] = res["step_us"] / res["empty_step_us"] if res.get("empty_step_us") else None
-        res["what"] = ("per timestep, measured by the library (lstm_probe): empty_step = publish -> L2 -> poll + CTA barrier, "
+        res["what"] = ("per timestep = recurrent launch / T, prologue included; step_us: the production kernel with the projection as its own "
+                       "launch; the rest measured by the library's probe builds (lstm_probe): empty_step = publish -> L2 -> poll + CTA barrier, "
                        "no products, no gate functions; compute_only = products + barrier + reduction + gates + stores without "
                        "waiting for other CTAs; the weights are read from the register file, so no shared-memory or HBM "
                        "bandwidth bounds the step: the exchange latency does")
