@@ -109,6 +109,8 @@ typedef struct {
  *                           to 40 steps on the register-resident kernel do so by default)
  *   LSTM_B200_WAVE  = 0     one launch per layer even where the layer-wavefront kernel would serve the stack
  *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
+ *   LSTM_B200_TC_ISSUE = 1|2  fewer issuing threads (and accumulators) in the batched tensor-core recurrence than the
+ *                           three it uses where the K extent allows
  *   LSTM_B200_COMPACT = 0   keep row/column-pruned units as explicit zeros, = 1 always run on the surviving units
  *                           (unset: handles with max_B >= 5 compact, smaller ones keep the zeros; see below)
  * Row/column-pruned stacks (Section 4.2, Algorithm 1: whole rows and columns of the gate matrices are zero).
@@ -240,7 +242,8 @@ LSTM_API int lstm_probe(lstm_handle *h, int parts_left_out);
  * (tcgen05) kernel, [8] kernels launched by the most recent lstm_forward (before the first call: the count expected),
  * [9] 1 if the recurrence keeps its weights in registers (bf16 dense), 0 for the shared-memory kernel,
  * [10] 16-column weight tiles per warp held in registers, [11] per warp held in shared memory,
- * [12] 1 if a call at max_B runs the batched tensor-core (tcgen05) recurrence: bf16 dense LSTM handles use
+ * [12] nonzero if a call at max_B runs the batched tensor-core (tcgen05) recurrence (2: as clusters of two CTAs
+ * that split K, 1: every CTA on its own): bf16 dense LSTM handles use
  * it for batches of 5 to 64 sequences where its operand ring fits beside the resident slice, and the
  * register-resident kernel (passes of four sequences) otherwise,
  * [13] 1 if a CSR handle runs the register-resident sparse kernel (bf16 storage, at most 16 units per CTA,

@@ -542,7 +542,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         const int RA = round_up(4 * h->upc, 8), nkb = (H + 63) / 64;
         if (!(bf16 && !csr && max_B > 4 && RA <= 128) || (env && (strcmp(env, "mma") == 0 || strcmp(env, "simt") == 0))) return false;
         const int B = std::min(max_B, 32), N = round_up(2 * B, 16);
-        return h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - 256, 0, kbs, stages);
+        return h->ncta_dir <= 160 && recur_tc_plan(RA, nkb, N, h->upc, B, (size_t)h->smem_optin - kTcStaticSmem, 0, kbs, stages);
     };
     int kbs_tmp = 0, stages_tmp = 0;
     if (D == 2 && bf16 && !csr && !h->use_mma && !tcb_fits(&kbs_tmp, &stages_tmp)) {
@@ -565,11 +565,17 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         const char *env = getenv("LSTM_B200_RECUR");
         const int Bp = std::min(max_B, 32), Np = round_up(2 * Bp, 16);
         int kp = 0, sp = 0;
+        // a pair's tile holds both CTAs' rows back to back: 2 x 4 x units is already a multiple of the 8-row swizzle
+        // group, so the rows are not padded (at 11 units per CTA the 8 rows saved per K block let the ring hold a
+        // whole step's operand)
+        const int RAp = 4 * h->upc;
         if (!(env && strcmp(env, "tc1") == 0) && (h->ncta_dir % 2) == 0 &&
-            recur_tc_plan(h->tcb_RA, h->tcb_nkb, Np, h->upc, Bp, (size_t)h->smem_optin - 256, 1, &kp, &sp) &&
-            recur_tc_prepare(h->smem_optin - 256) == cudaSuccess &&
-            recur_tc_pair_supported(h->ncta_dir * (h->seq_dirs ? 1 : D), recur_tc_smem_bytes(h->tcb_RA, h->tcb_nkb, Np, sp, kp, h->upc, Bp, 1)))
+            recur_tc_plan(RAp, h->tcb_nkb, Np, h->upc, Bp, (size_t)h->smem_optin - kTcStaticSmem, 1, &kp, &sp) &&
+            recur_tc_prepare(h->smem_optin - kTcStaticSmem) == cudaSuccess &&
+            recur_tc_pair_supported(h->ncta_dir * (h->seq_dirs ? 1 : D), recur_tc_smem_bytes(RAp, h->tcb_nkb, Np, sp, kp, h->upc, Bp, 1))) {
             h->tcb_pair = true;
+            h->tcb_RA = RAp;
+        }
     }
     h->layers.resize(layers);
     if (const char *env = getenv("LSTM_B200_SPIN_LIMIT")) { long long v = atoll(env); if (v > 0) h->spin_limit = v; }
@@ -810,7 +816,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                                          : recur_dense_prepare(h->smem_optin - 64);
         if (e == cudaSuccess && h->use_tc) e = proj_tc_prepare();
         if (e == cudaSuccess && csr) e = proj_csr_prepare(h->smem_optin - 64);
-        if (e == cudaSuccess && h->use_tcb) e = recur_tc_prepare(h->smem_optin - 256);
+        if (e == cudaSuccess && h->use_tcb) e = recur_tc_prepare(h->smem_optin - kTcStaticSmem);
         if (e != cudaSuccess) rc = fail(h, LSTM_ERR_CUDA, "kernel set-up failed: %s", cudaGetErrorString(e));
     }
     if (rc == LSTM_OK && cudaStreamSynchronize(st) != cudaSuccess)
@@ -1298,7 +1304,7 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         // (the plan made at create time covers up to 32 sequences; larger batches may not fit and then run as
         // passes of four on the kernels below)
         if (h->use_tcb && B > 4 && B <= kTcMaxBatch &&
-            recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * B, 16), h->upc, B, (size_t)h->smem_optin - 256, h->tcb_pair ? 1 : 0, &tc_kbs, &tc_stages)) {
+            recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * B, 16), h->upc, B, (size_t)h->smem_optin - kTcStaticSmem, h->tcb_pair ? 1 : 0, &tc_kbs, &tc_stages)) {
             RecurTcArgs m;
             memset(&m, 0, sizeof m);
             m.dir0 = h->seq_dirs ? pass : 0; m.ndirs = h->seq_dirs ? 1 : D;
@@ -1306,7 +1312,18 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.RA = h->tcb_RA; m.nkb = h->tcb_nkb; m.N = round_up(2 * B, 16);
             m.pair = h->tcb_pair ? 1 : 0;
             m.kbs = tc_kbs; m.stages = tc_stages;
-            m.tmem_cols = m.N <= 32 ? 32 : m.N <= 64 ? 64 : 128;
+            {
+                // issuing threads: as many as the smaller K share of a CTA allows, at most three
+                const int nkb_min = m.pair ? m.nkb / 2 : m.nkb;
+                int ni = nkb_min >= 3 ? 3 : nkb_min >= 2 ? 2 : 1;
+                if (const char *e = getenv("LSTM_B200_TC_ISSUE")) {
+                    const int want = atoi(e);
+                    if (want >= 1 && want <= ni) ni = want;
+                }
+                m.nissue = ni;
+                const int cols = ni * m.N;
+                m.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
+            }
             m.ldh = h->tcb_ldh;
             m.stamp_base = h->stamp_next;
             h->stamp_next += (unsigned)T + 1u;
@@ -1323,10 +1340,10 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
             m.hbuf = h->hplanes; m.flags = h->tcb_flags;
             m.status = h->status_dev;
-            if (h->tcb_mapN != m.N) {
-                if (!recur_tc_encode_planes(h->tmap_planes, h->hplanes, D, H, h->tcb_ldh, m.N))
+            if (h->tcb_mapN != B) {
+                if (!recur_tc_encode_planes(h->tmap_planes, h->hplanes, D, H, h->tcb_ldh, B))
                     return fail(h, LSTM_ERR_CUDA, "tensor map of the h planes could not be encoded");
-                h->tcb_mapN = m.N;
+                h->tcb_mapN = B;
             }
             const size_t smem = recur_tc_smem_bytes(m.RA, m.nkb, m.N, m.stages, m.kbs, h->upc, B, m.pair);
             if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
@@ -1600,8 +1617,8 @@ int lstm_info(const lstm_handle *h, int64_t *out, int n)
     const int launches = h->last_launches > 0 ? h->last_launches : h->L * 2 + (h->use_tc ? 1 : 0);
     int ik = 0, is = 0;
     const int tcb_at_max = (h->use_tcb && !h->Hh && h->max_B > 4 && h->max_B <= kTcMaxBatch &&
-                            recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * h->max_B, 16), h->upc, h->max_B, (size_t)h->smem_optin - 256,
-                                          h->tcb_pair ? 1 : 0, &ik, &is)) ? 1 : 0;
+                            recur_tc_plan(h->tcb_RA, h->tcb_nkb, round_up(2 * h->max_B, 16), h->upc, h->max_B, (size_t)h->smem_optin - kTcStaticSmem,
+                                          h->tcb_pair ? 1 : 0, &ik, &is)) ? (h->tcb_pair ? 2 : 1) : 0;
     if (h->use_csr_reg) shp.smem = recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, h->max_B);
     const int64_t vals[19] = {h->sm_count, h->ncta_dir, h->use_mma ? h->mma_nw * 32 : h->use_csr_reg ? h->csr_nw * 32 : h->threads, (int64_t)shp.smem,
                               rows_res, rows_str, (l0.plan_M >= 0) ? l0.plan.nsplit : 1, h->use_tc ? 1 : 0, launches,

@@ -185,6 +185,7 @@ cudaError_t launch_recur_csr_reg(const RecurCsrArgs &a, int slots, int nw, size_
 // 2b+1 = lo part of batch row b) and one stamp per producer CTA.
 // ---------------------------------------------------------------------------------------------------
 constexpr int kTcMaxBatch = 64;       // sequences per call the batched tensor-core recurrence serves
+constexpr int kTcStaticSmem = 1024;   // bytes kept free for the kernel's static shared memory (barriers, flags: under 600)
 constexpr int kTcPlaneRows = 128;     // rows of one parity of the h planes: hi and lo row of every sequence
 struct RecurTcArgs {
     int dir0, ndirs;            // directions this launch runs: dir0 .. dir0 + ndirs - 1 (ndirs = 0 means all D)
@@ -196,7 +197,8 @@ struct RecurTcArgs {
     int stages;                 // depth of the operand ring
     int kbs;                    // K blocks per ring stage
     int pair;                   // 1: clusters of two CTAs split K (launched with cluster dimension 2)
-    int tmem_cols;              // power of two >= max(32, N)
+    int nissue;                 // threads issuing tensor instructions, each with its own accumulator: 1 to 3, <= K blocks of any CTA
+    int tmem_cols;              // power of two >= max(32, nissue * N)
     int ldh;                    // row stride of the planes (elements, multiple of 8)
     unsigned stamp_base;
     long long spin_limit;
@@ -217,7 +219,7 @@ size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc,
 bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int pair, int *kbs_out, int *stages_out);
 bool recur_tc_pair_supported(int grid, size_t smem);
 bool recur_tc_encode_weights(void *map128, const void *w, long long rows, int ld, int RA);
-bool recur_tc_encode_planes(void *map128, const void *hbuf, int D, int H, int ldh, int N);
+bool recur_tc_encode_planes(void *map128, const void *hbuf, int D, int H, int ldh, int B);
 cudaError_t recur_tc_prepare(int max_smem);
 cudaError_t launch_recur_tc(const void *tmap_w, const void *tmap_h, const RecurTcArgs &a, size_t smem, cudaStream_t st);
 

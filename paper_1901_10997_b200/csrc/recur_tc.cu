@@ -14,19 +14,26 @@
 //   warp 0   waits until its own CTA has published the previous step, polls one stamp per producer CTA
 //            (relaxed loads, all in flight together, one fence after the last; bounded), then streams the
 //            [2B x H] operand into a ring of shared-memory stages with TMA (up to four 64-column blocks per
-//            stage, one issuing lane per block, zero fill at the tail);
-//   warp 1   issues M = 128, N = 2B (rounded up to 16), K = 16 tcgen05.mma instructions into one TMEM
-//            accumulator; the weight tile has only 4*units (<= 128) real rows: the rows beyond read whatever
-//            follows in shared memory and produce accumulator rows nobody reads;
-//   warps 2-5 request their projection terms, then read the accumulator rows of the CTA's units back
-//            (tcgen05.ld), add hi and lo columns, and finish the (unit, batch row) pairs: gates, c/h update,
-//            outputs, and the new h as bf16 planes; then one thread fences and raises the CTA's stamp.
+//            stage, one issuing lane per block, zero fill at the tail).  Every CTA (pair) reads the whole
+//            operand from L2, 148 SMs at once: this fetch, about 20 bytes per clock and SM, is the longest
+//            single part of a step;
+//   warps 1-3 issue M = 128, N = 2B (rounded up to 16), K = 16 tcgen05.mma instructions.  One thread issues
+//            such an instruction every 70 cycles or so whatever its shape, while the tensor cores finish it
+//            in far less at these N, so the K blocks are dealt round-robin to up to three issuing threads in
+//            three warps, each with a TMEM accumulator of its own (measured for 48 instructions: 3400
+//            cycles from one thread, 2340 from two, 1410 from four).  The weight tile has only 4*units
+//            (<= 128) real rows: the rows beyond read whatever follows in shared memory and produce
+//            accumulator rows nobody reads;
+//   warps 4-7 request their projection terms, then read the accumulator rows of the CTA's units back
+//            (tcgen05.ld), add the issuers' accumulators and the hi and lo columns, and finish the (unit,
+//            batch row) pairs: gates, c/h update, outputs, and the new h as bf16 planes; then one thread
+//            fences and raises the CTA's stamp.
 // Pair mode (chosen at create time when the CTA count per direction is even, the doubled tile fits and the
 // device can co-schedule the clusters): CTAs 2p and 2p+1 are launched as a cluster of two; each keeps the
 // weight rows of BOTH CTAs' units but only half of the K blocks, so each issues half the tensor
-// instructions per step; the partial sums of the partner's units go to the partner's shared memory
-// (st.shared::cluster) followed by a release arrive on the partner's mbarrier, and every CTA finishes its
-// own units from its own and the received partial sums.  The wait for the partner is bounded like the rest,
+// instructions per step; the partial sums of the partner's units are collected in shared memory and
+// sent to the partner's with one bulk copy (cp.async.bulk shared::cta -> shared::cluster) that completes on the
+// partner's mbarrier, and every CTA finishes its own units from its own and the received partial sums.  The wait for the partner is bounded like the rest,
 // and a cluster barrier at the common exit keeps a CTA resident while its partner may still write into it.
 // Every wait (stamps, mbarriers) is bounded; on expiry the CTA records a timeout status and all roles fall
 // through to the common exit where tensor memory is released.  No TMA multicast is used.
@@ -40,12 +47,12 @@
 namespace lstm {
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 256;                  // producer warp, three issuing warps, four finishing warps
+constexpr int kFinishTid0 = 128;                // first thread of the finishing warps
 constexpr int kMaxStages = 8;
 constexpr int kFlagLoads = 5;                   // stamps one lane polls: up to 160 CTAs per direction
 constexpr int kPre = 2;                         // (unit, batch row) items per thread whose projection terms are prefetched
 constexpr int kMaxSplit = 4;                    // split-K partial sums of the projection
-constexpr long long kWaitTicks = kMbarWaitTicks;
 
 // ---- two-CTA cluster helpers (pair mode): the partner's shared memory and barriers
 __device__ __forceinline__ uint32_t cluster_ctarank()
@@ -60,39 +67,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v)
+// shared memory of this CTA -> shared memory of another CTA of the cluster (addresses and size multiples of 16
+// bytes); the bytes are counted on the destination CTA's barrier
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t remote_dst, uint32_t local_src, uint32_t bytes, uint32_t remote_bar)
 {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t remote_bar)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_acquire_cluster(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait for the partner's arrival; false when it gave up or another role did.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    long long t_start = 0;
-    for (long long it = 0;; ++it) {
-        if (mbar_try_wait_acquire_cluster(bar, parity)) return true;
-        if ((it & 255) == 255) {
-            if (*abort_flag) return false;
-            const long long now = clock64();
-            if (t_start == 0) t_start = now;
-            if (now - t_start > kWaitTicks) break;
-        }
-    }
-    *abort_flag = 1;
-    return false;
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(remote_dst), "r"(local_src), "r"(bytes), "r"(remote_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all()
 {
@@ -111,6 +91,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int H = a.H, B = a.B, T = a.T, D = a.D, N = a.N, S = a.stages, RA = a.RA, nkb = a.nkb, kbs = a.kbs;
+    const int NB = (2 * B + 7) & ~7;             // rows of a fetched operand block: the copy leaves out the rows that only pad N
     const int d = a.dir0 + blockIdx.x / a.ncta_dir;
     const int cta = blockIdx.x % a.ncta_dir;
     int u0, nu;
@@ -126,6 +107,8 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     const int kb_lo = (pair && rank) ? nkb_half : 0;                        // first K block of this CTA
     const int nkb_my = pair ? (rank ? nkb - nkb_half : nkb_half) : nkb;     // K blocks of this CTA
     const int nkb_alloc = pair ? nkb_half : nkb;                            // same layout in both CTAs of a pair
+    const int groups = (nkb_my + kbs - 1) / kbs;                            // ring stages one step's operand takes
+    const bool whole = groups <= S && nkb_my <= 32;                         // the ring holds it all: every step starts at stage 0
 
     // shared-memory carve-up (tiles need 1024-byte alignment): weight tiles, operand ring, then scratch
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -135,16 +118,17 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
     float *zs = reinterpret_cast<float *>(gen);                             // [B][4*upc] gate pre-activations (h part)
     const int zld = 4 * upc;
     float *c_s = zs + zld * B;                                              // [B][units of this CTA]
-    float *zs2 = c_s + ((upc * B + 3) & ~3);                                // [B][4*upc] the partner's partial sums (pair mode)
+    float *zs2 = c_s + ((upc * B + 3) & ~3);                                // [B][4*upc] partial sums received from the partner (pair mode)
+    float *zsp = zs2 + (pair ? zld * B : 0);                                // [B][4*upc] partial sums of the partner's units, before they are sent
     // checked build: the carve-up ends inside the launch's shared memory, and so does the 128-row read of the last weight tile
-    LSTM_CHECK_SMEM_END((size_t)(reinterpret_cast<unsigned char *>(zs2 + (pair ? zld * B : 0)) - smem_raw), a.status);
+    LSTM_CHECK_SMEM_END((size_t)(reinterpret_cast<unsigned char *>(zsp + (pair ? zld * B : 0)) - smem_raw), a.status);
     LSTM_CHECK_SMEM_END((size_t)(a_tiles - smem_u32(smem_raw)) + (size_t)(nkb_alloc - 1) * RT * 128 + (size_t)128 * 128, a.status);
 
     if (tid == 0) {
         abort_s = 0;
         pub_s = 0;
-        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-        mbar_init(smem_u32(&accum_bar), 1);
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), (uint32_t)a.nissue); }
+        mbar_init(smem_u32(&accum_bar), (uint32_t)a.nissue);
         mbar_init(smem_u32(&w_bar), 1);
         mbar_init(smem_u32(&partial_bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -198,7 +182,8 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             }
             __syncwarp();
             // every producer's stamp of the previous step (the prologue publishes h0 with stamp_base): relaxed
-            // loads, all in flight together, and one fence once they all show the stamp
+            // loads, all in flight together, and one fence once they all show the stamp (acquire loads in the
+            // polling loop were measured far slower)
             const unsigned want = a.stamp_base + (unsigned)s;
             long long t_start = 0;
             int rounds = 0;
@@ -230,14 +215,28 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             }
             if (aborted) break;
             fence_acq_rel_gpu();                                    // acquire: the planes behind the stamps
-            asm volatile("fence.proxy.async;" ::: "memory");       // they were written with ordinary stores
+            asm volatile("fence.proxy.async.global;" ::: "memory");    // they were written with ordinary stores
             const int row0 = (d * 2 + ((s + 1) & 1)) * kTcPlaneRows;   // planes of step s-1 live in parity (s-1)&1
+            if (whole) {
+                // the ring holds the whole operand (every step starts at stage 0 with the same phase): lane i < groups
+                // opens stage i, then one lane per K block issues its copy, all in the same instruction
+                int ok = 1;
+                if (lane < groups) {
+                    const int nblk = min(kbs, nkb_my - lane * kbs);
+                    ok = mbar_wait(smem_u32(&empty_bar[lane]), ((uint32_t)s & 1u) ^ 1u, abort_flag) ? 1 : 0;
+                    if (ok) mbar_expect_tx(smem_u32(&full_bar[lane]), (uint32_t)(nblk * NB) * 128);
+                }
+                if (!__all_sync(0xffffffffu, ok)) break;
+                if (lane < nkb_my)
+                    tma_load_2d(ring + (uint32_t)(lane * N) * 128, &tmap_h, smem_u32(&full_bar[lane / kbs]), (kb_lo + lane) * 64, row0);
+                continue;
+            }
             for (int g0 = 0; g0 < nkb_my; g0 += kbs) {
                 const int nblk = min(kbs, nkb_my - g0);
                 int ok = 1;
                 if (lane == 0) {
                     ok = mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abort_flag) ? 1 : 0;
-                    if (ok) mbar_expect_tx(smem_u32(&full_bar[st]), (uint32_t)(nblk * N) * 128);
+                    if (ok) mbar_expect_tx(smem_u32(&full_bar[st]), (uint32_t)(nblk * NB) * 128);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { live = false; break; }
@@ -247,28 +246,39 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                 if (++st == S) { st = 0; ph ^= 1u; }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp <= 3) {
         // ================= MMA issue =================
-        if (lane == 0) {
+        // issuer w = warp - 1 < nissue takes the K blocks whose index is w modulo nissue (no CTA has fewer K blocks
+        // than issuers) into the accumulator at TMEM column w * N; every issuer passes every stage and commits to
+        // its barriers, blocks or not
+        const int w = warp - 1;
+        if (lane == 0 && w < a.nissue) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
             bool ok = mbar_wait(smem_u32(&w_bar), 0u, abort_flag);
             // descriptors differ only in their start-address field (units of 16 bytes): build one of each and add
             const uint64_t adesc0 = umma_desc_sw128(a_tiles), bdesc0 = umma_desc_sw128(ring);
             const uint32_t a_step = (uint32_t)(RT * 128) >> 4, b_step = (uint32_t)(N * 128) >> 4;
+            const uint32_t acc = tmem_base + (uint32_t)(w * N);
             int st = 0;
             uint32_t ph = 0;
             for (int s = 0; s < T && ok; ++s) {
-                uint64_t adesc = adesc0;
+                uint32_t accumulate = 0u;
+                int next = w;                                   // this issuer's next K block
+                if (whole) { st = 0; ph = (uint32_t)s & 1u; }
                 for (int g0 = 0; g0 < nkb_my; g0 += kbs) {
                     const int nblk = min(kbs, nkb_my - g0);
                     ok = mbar_wait(smem_u32(&full_bar[st]), ph, abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)(st * kbs) * b_step);
-                    for (int l = 0; l < nblk; ++l, adesc += a_step, bdesc += b_step) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (g0 + l > 0 || k > 0) ? 1u : 0u);
+                    for (; next < g0 + nblk; next += a.nissue) {
+                        const int l = next - g0;
+                        const uint64_t adesc = adesc0 + (uint64_t)((uint32_t)(g0 + l) * a_step);
+                        const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)(st * kbs + l) * b_step);
+                        umma_bf16(acc, adesc, bdesc, idesc, accumulate);
+                        umma_bf16(acc, adesc + 2, bdesc + 2, idesc, 1u);
+                        umma_bf16(acc, adesc + 4, bdesc + 4, idesc, 1u);
+                        umma_bf16(acc, adesc + 6, bdesc + 6, idesc, 1u);
+                        accumulate = 1u;
                     }
                     umma_commit(smem_u32(&empty_bar[st]));
                     if (++st == S) { st = 0; ph ^= 1u; }
@@ -278,7 +288,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
         }
     } else {
         // ================= accumulator read-back and the cell =================
-        const int ftid = tid - 64;                       // 0..127
+        const int ftid = tid - kFinishTid0;              // 0..127
         const int lq = warp & 3;                         // TMEM lane quadrant this warp may read
         const int nuB = nu * B;
         int u0_partner = 0, nu_partner = 0;
@@ -306,6 +316,14 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             *pub = 1;
         }
         const size_t gs4 = (size_t)(a.g_split_stride / 4);
+        // the first kPre items of this thread: batch row and unit, fixed for the whole sequence
+        int pb[kPre], pu[kPre];
+#pragma unroll
+        for (int i = 0; i < kPre; ++i) {
+            const int p = ftid + 128 * i;
+            pb[i] = p < nuB ? p / nu : 0;
+            pu[i] = p < nuB ? p - pb[i] * nu : 0;
+        }
         for (int s = 0; s < T; ++s) {
             const int t = d ? (T - 1 - s) : s;
             // projection terms of the first items: requested before the wait, they do not depend on h
@@ -314,7 +332,7 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             for (int i = 0; i < kPre; ++i) {
                 const int p = ftid + 128 * i;
                 if (p < nuB) {
-                    const int b = p / nu, j = u0 + p - b * nu;
+                    const int b = pb[i], j = u0 + pu[i];
                     const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)j * 4);
 #pragma unroll
                     for (int sp = 0; sp < kMaxSplit; ++sp)
@@ -335,11 +353,24 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                 // one wait; batches above 32 read their remaining chunks one at a time (registers)
                 const int nchunk = (2 * B + 15) >> 4;
                 {
-                    uint32_t v[4][16];
+                    float z[4][8];
+                    // one issuer's accumulator after the other; hi and lo columns are added on the way
+                    for (int wi = 0; wi < a.nissue; ++wi) {
+                        uint32_t x[4][16];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (c < nchunk) tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(c * 16), v[c]);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        for (int c = 0; c < 4; ++c)
+                            if (c < nchunk) tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(wi * N + c * 16), x[c]);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            if (c < nchunk) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const float zz = __uint_as_float(x[c][2 * i]) + __uint_as_float(x[c][2 * i + 1]);
+                                    z[c][i] = wi ? z[c][i] + zz : zz;
+                                }
+                            }
+                    }
                     if (row_ok) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
@@ -347,10 +378,8 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) {
                                     const int b = c * 8 + i;
-                                    const float z = __uint_as_float(v[c][2 * i]) + __uint_as_float(v[c][2 * i + 1]);
                                     if (b < B) {
-                                        if (mine) zs[b * zld + lr] = z;
-                                        else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                                        (mine ? zs : zsp)[b * zld + lr] = z[c][i];
                                     }
                                 }
                             }
@@ -362,14 +391,20 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                     uint32_t w[16];
                     tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(c * 16), w);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    for (int wi = 1; wi < a.nissue; ++wi) {
+                        uint32_t x[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(lq * 32) << 16) + (uint32_t)(wi * N + c * 16), x);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) + __uint_as_float(x[i]));
+                    }
                     if (row_ok) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const int b = c * 8 + i;
                             const float z = __uint_as_float(w[2 * i]) + __uint_as_float(w[2 * i + 1]);
                             if (b < B) {
-                                if (mine) zs[b * zld + lr] = z;
-                                else st_cluster_f32(zs2_remote + (uint32_t)(b * zld + lr) * 4u, z);
+                                (mine ? zs : zsp)[b * zld + lr] = z;
                             }
                         }
                     }
@@ -378,31 +413,20 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             bar_sync(1, 128);
             if (pair) {
-                // tell the partner its partial sums are in place, then wait for ours (bounded)
-                if (ftid == 0) mbar_arrive_remote_release(partial_bar_remote);
-                if (!mbar_wait_cluster(smem_u32(&partial_bar), (uint32_t)s & 1u, abort_flag)) break;
+                // one bulk copy carries the partner's partial sums into its shared memory and completes on its
+                // barrier; ours arrive the same way (bounded wait)
+                if (ftid == 0) {
+                    const uint32_t bytes = (uint32_t)(zld * B) * 4u;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_expect_tx(smem_u32(&partial_bar), bytes);
+                    bulk_copy_to_cta(zs2_remote, smem_u32(zsp), bytes, partial_bar_remote);
+                }
+                if (!mbar_wait(smem_u32(&partial_bar), (uint32_t)s & 1u, abort_flag)) break;
             }
             __nv_bfloat16 *hp = hbuf_d + (size_t)(s & 1) * kTcPlaneRows * a.ldh;
-            for (int i = 0; ftid + 128 * i < nuB; ++i) {
-                const int p = ftid + 128 * i;
-                const int b = p / nu, u = p - b * nu, j = u0 + u;       // consecutive threads, consecutive units
-                float4 gsum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                if (i < kPre) {
-#pragma unroll
-                    for (int ii = 0; ii < kPre; ++ii) {
-                        if (ii == i) {
-#pragma unroll
-                            for (int sp = 0; sp < kMaxSplit; ++sp)
-                                if (sp < a.nsplit) { gsum.x += gpre[ii][sp].x; gsum.y += gpre[ii][sp].y; gsum.z += gpre[ii][sp].z; gsum.w += gpre[ii][sp].w; }
-                        }
-                    }
-                } else {
-                    const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)j * 4);
-                    for (int sp = 0; sp < a.nsplit; ++sp) {
-                        const float4 g4 = __ldg(gp + (size_t)sp * gs4);
-                        gsum.x += g4.x; gsum.y += g4.y; gsum.z += g4.z; gsum.w += g4.w;
-                    }
-                }
+            // one (unit, batch row) item: gates, c/h update, the new h as planes, outputs
+            auto finish_item = [&](int p, int b, int u, const float4 &gsum) {
+                const int j = u0 + u;
                 float4 z4 = *reinterpret_cast<const float4 *>(zs + b * zld + 4 * u);
                 if (pair) {
                     const float4 y4 = *reinterpret_cast<const float4 *>(zs2 + b * zld + 4 * u);
@@ -429,12 +453,33 @@ recur_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constan
                     if (a.hT) a.hT[((size_t)d * B + b) * H + j] = hn;
                     if (a.cT) a.cT[((size_t)d * B + b) * H + j] = cn;
                 }
+            };
+            // consecutive threads, consecutive units; the first kPre items have their projection terms in registers
+#pragma unroll
+            for (int i = 0; i < kPre; ++i) {
+                const int p = ftid + 128 * i;
+                if (p < nuB) {
+                    float4 gsum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+                    for (int sp = 0; sp < kMaxSplit; ++sp)
+                        if (sp < a.nsplit) { gsum.x += gpre[i][sp].x; gsum.y += gpre[i][sp].y; gsum.z += gpre[i][sp].z; gsum.w += gpre[i][sp].w; }
+                    finish_item(p, pb[i], pu[i], gsum);
+                }
+            }
+            for (int p = ftid + 128 * kPre; p < nuB; p += 128) {
+                const int b = p / nu, u = p - b * nu;
+                const float4 *gp = reinterpret_cast<const float4 *>(a.G + (((size_t)t * B + b) * D + d) * 4 * H + (size_t)(u0 + u) * 4);
+                float4 gsum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                for (int sp = 0; sp < a.nsplit; ++sp) {
+                    const float4 g4 = __ldg(gp + (size_t)sp * gs4);
+                    gsum.x += g4.x; gsum.y += g4.y; gsum.z += g4.z; gsum.w += g4.w;
+                }
+                finish_item(p, b, u, gsum);
             }
             bar_sync(1, 128);
             if (ftid == 0) {
                 if ((int)blockIdx.x != a.withhold_cta) {
-                    fence_acq_rel_gpu();
-                    st_relaxed_u32(flags_d + cta, a.stamp_base + (unsigned)s + 1u);
+                    st_release_u32(flags_d + cta, a.stamp_base + (unsigned)s + 1u);
                 }
                 *pub = s + 2;
             }
@@ -465,18 +510,28 @@ size_t recur_tc_smem_bytes(int RA, int nkb, int N, int stages, int kbs, int upc,
     // pair mode: tiles of 2 RA rows, half of the K blocks (rounded up), and a second block of partial sums
     const int RT = pair ? 2 * RA : RA, nkb_alloc = pair ? (nkb + 1) / 2 : nkb;
     // the last weight tile is read as 128 rows: at least (128 - RT) * 128 bytes must follow it
-    const size_t scratch = (size_t)(4 * upc * B) * (pair ? 2 : 1) + (size_t)((upc * B + 3) & ~3);
+    const size_t scratch = (size_t)(4 * upc * B) * (pair ? 3 : 1) + (size_t)((upc * B + 3) & ~3);
     const size_t after = (size_t)stages * kbs * N * 128 + scratch * 4 + 16;
     const size_t need = (size_t)(128 - RT) * 128;
     return 1024 + (size_t)nkb_alloc * RT * 128 + (after > need ? after : need);
 }
 
 // Ring shape for one launch: stages of up to four K blocks (one mbarrier round trip per stage instead of per
-// block), as many stages as fit, at least two unless one stage holds the whole operand.
+// block); a ring that holds the whole operand if one fits, else as many stages as fit, at least two.
 bool recur_tc_plan(int RA, int nkb, int N, int upc, int B, size_t max_smem, int pair, int *kbs_out, int *stages_out)
 {
     const int nkb_cta = pair ? (nkb + 1) / 2 : nkb;
     if (pair && (2 * RA > 128 || nkb < 2)) return false;
+    // first choice: a ring that holds a whole step's operand (all copies of a step are then issued together),
+    // in as few stages as possible
+    for (int kbs = nkb_cta < 4 ? nkb_cta : 4; kbs >= 1 && nkb_cta <= 32; --kbs) {
+        const int st = (nkb_cta + kbs - 1) / kbs;
+        if (st <= kMaxStages && recur_tc_smem_bytes(RA, nkb, N, st, kbs, upc, B, pair) <= max_smem) {
+            *kbs_out = kbs;
+            *stages_out = st;
+            return true;
+        }
+    }
     for (int kbs = nkb_cta < 4 ? nkb_cta : 4; kbs >= 1; --kbs) {
         const int groups = (nkb_cta + kbs - 1) / kbs;
         for (int st = groups < kMaxStages ? groups : kMaxStages; st >= (groups > 1 ? 2 : 1); --st) {
@@ -494,9 +549,10 @@ bool recur_tc_encode_weights(void *map, const void *w, long long rows, int ld, i
 {
     return encode_2d(map, w, rows, ld, ld, RA);
 }
-bool recur_tc_encode_planes(void *map, const void *hbuf, int D, int H, int ldh, int N)
+bool recur_tc_encode_planes(void *map, const void *hbuf, int D, int H, int ldh, int B)
 {
-    return encode_2d(map, hbuf, (long long)D * 2 * kTcPlaneRows, H, ldh, N);
+    // a box holds the 2B plane rows rounded up to a swizzle group of 8, not the MMA's N (a multiple of 16)
+    return encode_2d(map, hbuf, (long long)D * 2 * kTcPlaneRows, H, ldh, (2 * B + 7) & ~7);
 }
 
 cudaError_t recur_tc_prepare(int max_smem)

@@ -232,7 +232,7 @@ def test_batched_tensor_core_recurrence(oracle, w):
     h0, c0 = wl.make_states(w)
     ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
     m = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype="bf16", max_T=w.T, max_B=w.B)
-    assert m.info()["recur_batched_tensor_core"] == (0 if w.name.startswith("notc") else 1)
+    assert bool(m.info()["recur_batched_tensor_core"]) == (not w.name.startswith("notc"))
     y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
     m.check()
     assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", w.name)
@@ -259,7 +259,7 @@ def test_first_call_of_a_fresh_handle_sees_a_nonzero_initial_state(oracle, B):
     ref = oracle.forward(weights, x, h0, c0, layers=1, bidir=False, hidden=w.hidden)
     for _ in range(4):
         m = pkg.LSTM(weights, layers=1, in_dim=w.in_dim, hidden=w.hidden, dtype="bf16", max_T=w.T, max_B=w.B)
-        assert m.info()["recur_batched_tensor_core"] == 1
+        assert m.info()["recur_batched_tensor_core"] >= 1
         y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
         m.check()
         assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"fresh handle B={B}")
