@@ -311,6 +311,7 @@ struct ProjTcPlan {
     int n_tile;        // MMA N extent (activation rows per tile), multiple of 16, <= 256
     int nsplit;        // split-K factor
     int kblocks;       // ceil(K / 64)
+    int sm_count;      // CTAs of the persistent kernel that serves shapes with several activation tiles
 };
 int  proj_tc_plan(ProjTcPlan *p, const __nv_bfloat16 *W, const __nv_bfloat16 *X, const __nv_bfloat16 *Xlo,
                   int M, int N, int K, int ldk, int sm_count, char *err, int errlen);
