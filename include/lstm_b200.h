@@ -109,6 +109,8 @@ typedef struct {
  *                           to 40 steps on the register-resident kernel do so by default)
  *   LSTM_B200_WAVE  = 0     one launch per layer even where the layer-wavefront kernel would serve the stack
  *   LSTM_B200_PROJ  = simt  CUDA-core input projection instead of the tensor-core one
+ *                   = csr   CSR handles walk the lists of Wx in the projection too (by default bf16 CSR handles keep a
+ *                           dense copy of Wx and project on the tensor cores; the recurrence stays sparse)
  *   LSTM_B200_PROJ_TILE = 128  the 128-row-tile projection kernel (two CTAs per SM) also where the persistent
  *                           256-row-tile kernel would run (several activation tiles)
  *   LSTM_B200_PROJ_SMEM_KB = 48..200  shared-memory budget of the 128-row-tile projection kernel (ring depth)

@@ -60,6 +60,7 @@ struct lstm_handle {
     bool fuse_ok = false;              // short single sequences: projection fused into the register-resident kernel's prologue
     // register-resident sparse kernel (bf16, CSR execution): warps, columns per warp, row tiles, entry slots per lane
     bool use_csr_reg = false;
+    bool csr_dense_proj = false;       // CSR handle whose input projection runs on the tensor cores over Wx with explicit zeros
     int csr_nw = 0, csr_kspan = 0, csr_mt = 0, csr_slots = 0;
     long long csr_conflicts = 0;       // shared-memory wavefronts per step and CTA lost to bank conflicts (worst CTA, worst matrix)
     int mma_mt = 0, mma_nkr = 0, mma_nks = 0, mma_nw = 0;
@@ -518,6 +519,16 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
     h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
+    {
+        // A pruned Wx still makes a dense contraction with all timesteps as the other operand, and at the densities
+        // pruning reaches (0.05 .. 0.10) the tensor cores multiply the zeros faster than CUDA cores walk the lists
+        // (the paper's own observation about sparse matmuls on GPUs, Section 3): bf16 CSR handles keep a dense
+        // copy of Wx for the projection; the recurrence, where the lists stay on-chip, remains sparse.
+        // LSTM_B200_PROJ=csr keeps the list-walking projection, =simt the CUDA-core dense one.
+        const char *env = getenv("LSTM_B200_PROJ");
+        h->csr_dense_proj = csr && bf16 && !(env && (strcmp(env, "csr") == 0 || strcmp(env, "simt") == 0));
+        if (h->csr_dense_proj) h->use_tc = true;
+    }
     plan_mma(h);
     plan_wave(h);
     {
@@ -596,7 +607,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         std::vector<int> px_rowptr; std::vector<CsrEntry> px_ent;
         std::vector<uint16_t> tcb_rows;
         if (!csr) { if (bf16) wx16.assign((size_t)N * ly.ldk, 0); else wx32.assign((size_t)N * ly.ldk, 0.0f); }
-        else px_rowptr.assign(N + 1, 0);
+        else { px_rowptr.assign(N + 1, 0); if (h->csr_dense_proj) wx16.assign((size_t)N * ly.ldk, 0); }
 
         for (int d = 0; d < D && rc == LSTM_OK; ++d) {
             const lstm_weights &src = w[l * D + d];
@@ -704,6 +715,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                             float v = cx.val[e];
                             if (bf16) v = bf16_to_f32(f32_to_bf16_rne(v));
                             px_ent.push_back(CsrEntry{v, cx.col[e]});
+                            if (h->csr_dense_proj) wx16[((size_t)d * 4 * H + (size_t)j * 4 + q) * ly.ldk + cx.col[e]] = f32_to_bf16_rne(cx.val[e]);
                         }
                         px_rowptr[(size_t)d * 4 * H + (size_t)j * 4 + q + 1] = (int)px_ent.size();
                     }
@@ -749,6 +761,8 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         if (rc == LSTM_OK && !csr)
             rc = bf16 ? upload(h, (uint16_t **)&ly.wx, wx16.data(), wx16.size() * 2, st, "input weights")
                       : upload(h, (float **)&ly.wx, wx32.data(), wx32.size() * 4, st, "input weights");
+        if (rc == LSTM_OK && h->csr_dense_proj)
+            rc = upload(h, (uint16_t **)&ly.wx, wx16.data(), wx16.size() * 2, st, "input weights (dense copy)");
         if (rc == LSTM_OK && csr) {
             rc = upload(h, &ly.wx_rowptr, px_rowptr.data(), px_rowptr.size() * sizeof(int), st, "input CSR offsets");
             if (rc == LSTM_OK) rc = upload(h, &ly.wx_ent, px_ent.data(), px_ent.size() * sizeof(CsrEntry), st, "input CSR entries");
@@ -1125,7 +1139,7 @@ static int run_projection(lstm_handle *h, int l, const float *x, const float *Xf
     cudaError_t e = cudaSuccess;
     int nsplit = 1;
     // ---- input staging + projection
-    if (csr) {
+    if (csr && !h->csr_dense_proj) {
         if (record(h, LSTM_K_PROJ, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
         e = launch_proj_csr(Xf, ly.wx_rowptr, ly.wx_ent, ly.bias, h->G, M, N, ly.in_l, !bf16, st);
         ++h->last_launches;
@@ -1371,7 +1385,9 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
             m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
             m.y = l == L - 1 ? y : h->ybuf[l & 1];
-            m.xb_next = nullptr;
+            m.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
+            m.xb_ld = h->ldn;
+            m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
             m.xch = h->xch;
             m.status = h->status_dev;
             const size_t smem = recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, B);
