@@ -114,6 +114,7 @@ typedef struct {
  *   LSTM_B200_PROJ_TILE = 128  the 128-row-tile projection kernel (two CTAs per SM) also where the persistent
  *                           256-row-tile kernel would run (several activation tiles)
  *   LSTM_B200_PROJ_SMEM_KB = 48..200  shared-memory budget of the 128-row-tile projection kernel (ring depth)
+ *   LSTM_B200_CTAS  = <n>   at most n CTAs per direction in the recurrent kernels (measurement)
  *   LSTM_B200_TC_ISSUE = 1|2  fewer issuing threads (and accumulators) in the batched tensor-core recurrence than the
  *                           three it uses where the K extent allows
  *   LSTM_B200_COMPACT = 0   keep row/column-pruned units as explicit zeros, = 1 always run on the surviving units

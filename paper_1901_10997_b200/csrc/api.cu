@@ -516,7 +516,15 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
     h->Hp8 = round_up(H, 8);
     h->Hs = round_up(H, 256);
     h->ncta_dir = std::max(1, std::min(h->sm_count / D, H));
+    if (const char *e = getenv("LSTM_B200_CTAS")) {     // measurement: fewer CTAs per direction than SMs
+        const int want = atoi(e);
+        if (want >= 1 && want <= h->ncta_dir) h->ncta_dir = want;
+    }
     h->upc = (H + h->ncta_dir - 1) / h->ncta_dir;
+    // fp32 storage: no more CTAs than full slices (H = 200: 100 CTAs of two units, not 52 of two and 96 of one).
+    // The step waits for the slowest CTA either way, and every CTA less is B * H fewer words polled per step
+    // (workload 1: 6.8 -> 5.3 us per step).
+    if (dtype == LSTM_F32) h->ncta_dir = (H + h->upc - 1) / h->upc;
     h->threads = std::max(128, 32 * std::min(h->upc, 16));
     h->use_tc = want_tc(h);
     {

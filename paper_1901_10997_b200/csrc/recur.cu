@@ -34,6 +34,13 @@ __device__ __forceinline__ int h_pos(int k, int Hs)
     return k;
 }
 
+__device__ __forceinline__ float shfl_xor_at(float v, int o) { return __shfl_xor_sync(0xffffffffu, v, o); }
+__device__ __forceinline__ double shfl_xor_at(double v, int o) { return __shfl_xor_sync(0xffffffffu, v, o); }
+// arithmetic type of the gate functions and the state update, and the accumulator's value in it
+template <typename AT> struct GateOf { typedef AT T; };
+__device__ __forceinline__ float gate_value(float v) { return v; }
+__device__ __forceinline__ double gate_value(double v) { return v; }
+
 // Sum V values per lane over the 32 lanes of a warp.  On return lane l holds the total of value
 // index l >> (5 - log2 V).  Each halving step exchanges half of the remaining values, so V values cost
 // V - 1 + (5 - log2 V) shuffles instead of 5 V.
@@ -50,12 +57,12 @@ __device__ __forceinline__ AT warp_reduce_multi(AT (&v)[V], int lane)
         for (int k = 0; k < n / 2; ++k) {
             const AT send = upper ? v[k] : v[k + n / 2];
             const AT keep = upper ? v[k + n / 2] : v[k];
-            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            v[k] = keep + shfl_xor_at(send, o);
         }
         o >>= 1;
     }
 #pragma unroll
-    for (int o2 = (16 >> LOG2V); o2 >= 1; o2 >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], o2);
+    for (int o2 = (16 >> LOG2V); o2 >= 1; o2 >>= 1) v[0] += shfl_xor_at(v[0], o2);
     return v[0];
 }
 
@@ -99,12 +106,14 @@ __device__ __forceinline__ void unit_dot_dense(const WT *rows, int Hp8, const fl
             load_w8(rows + (size_t)q * Hp8, v8, w);
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
-                AT s = acc[q * BT + b];
-                s = fma((AT)w[0], (AT)hlo[b].x, s); s = fma((AT)w[1], (AT)hlo[b].y, s);
-                s = fma((AT)w[2], (AT)hlo[b].z, s); s = fma((AT)w[3], (AT)hlo[b].w, s);
-                s = fma((AT)w[4], (AT)hhi[b].x, s); s = fma((AT)w[5], (AT)hhi[b].y, s);
-                s = fma((AT)w[6], (AT)hhi[b].z, s); s = fma((AT)w[7], (AT)hhi[b].w, s);
-                acc[q * BT + b] = s;
+                // eight terms in fp32 (two chains of four; their rounding error is a few 1e-8 of the terms'
+                // size), the partial sums added up in AT: with a double or two-float AT the long sum over H
+                // stays exact to far below fp32 rounding
+                float s0 = w[0] * hlo[b].x, s1 = w[4] * hhi[b].x;
+                s0 = fmaf(w[1], hlo[b].y, s0); s1 = fmaf(w[5], hhi[b].y, s1);
+                s0 = fmaf(w[2], hlo[b].z, s0); s1 = fmaf(w[6], hhi[b].z, s1);
+                s0 = fmaf(w[3], hlo[b].w, s0); s1 = fmaf(w[7], hhi[b].w, s1);
+                acc[q * BT + b] += (AT)(s0 + s1);
             }
         }
     }
@@ -141,19 +150,20 @@ __device__ __forceinline__ void unit_dot_csr(const ET *ent, const int (&e)[5], c
         decode4(ent, vi, w, col);
 #pragma unroll
         for (int b = 0; b < BT; ++b) {
-            AT s = (AT)w[0] * (AT)hb[b * Hs + col[0]];
-            s = fma((AT)w[1], (AT)hb[b * Hs + col[1]], s);
-            s = fma((AT)w[2], (AT)hb[b * Hs + col[2]], s);
-            s = fma((AT)w[3], (AT)hb[b * Hs + col[3]], s);
+            float s = w[0] * hb[b * Hs + col[0]];
+            s = fmaf(w[1], hb[b * Hs + col[1]], s);
+            s = fmaf(w[2], hb[b * Hs + col[2]], s);
+            s = fmaf(w[3], hb[b * Hs + col[3]], s);
 #pragma unroll
-            for (int qq = 0; qq < 4; ++qq) acc[qq * BT + b] += (q == qq) ? s : (AT)0;
+            for (int qq = 0; qq < 4; ++qq) acc[qq * BT + b] += (AT)((q == qq) ? s : 0.0f);
         }
     }
 }
 
-// bf16 storage: fp32 accumulation and gate functions.  fp32 storage: dot products accumulate in fp64
-// and the gate functions are evaluated in fp64, so the only fp32 roundings left are the stored
-// projection, h and c -- what the 1e-4 agreement bound of that mode needs.
+// bf16 storage: fp32 accumulation and gate functions.  fp32 storage: short fp32 chains of four or eight terms
+// added up in fp64, and the gate functions and the state update in fp64, so the only fp32 roundings left are
+// the stored projection, h and c -- what the 1e-4 agreement bound of that mode needs (two-float sums with fp32
+// gate functions were measured: 1.02e-4 on the floored metric, and no faster: the step waits for the exchange).
 template <bool BF16> struct Types { typedef __nv_bfloat16 W; typedef unsigned E; typedef float A; };
 template <> struct Types<false> { typedef float W; typedef CsrEntry E; typedef double A; };
 
@@ -274,15 +284,16 @@ __global__ void __launch_bounds__(512, 1) recur_kernel(const RecurArgs a)
             }
         }
         z += (AT)g_in;
-        const AT act = gate_fn(z, q_mine == 2);
-        const AT vi = __shfl_sync(0xffffffffu, act, (0 * BT + b_gather) << SH);
-        const AT vf = __shfl_sync(0xffffffffu, act, (1 * BT + b_gather) << SH);
-        const AT vg = __shfl_sync(0xffffffffu, act, (2 * BT + b_gather) << SH);
-        const AT vo = __shfl_sync(0xffffffffu, act, (3 * BT + b_gather) << SH);
+        typedef typename GateOf<AT>::T GT;
+        const GT act = gate_fn(gate_value(z), q_mine == 2);
+        const GT vi = __shfl_sync(0xffffffffu, act, (0 * BT + b_gather) << SH);
+        const GT vf = __shfl_sync(0xffffffffu, act, (1 * BT + b_gather) << SH);
+        const GT vg = __shfl_sync(0xffffffffu, act, (2 * BT + b_gather) << SH);
+        const GT vo = __shfl_sync(0xffffffffu, act, (3 * BT + b_gather) << SH);
         if (lane < nb) {
             const int b = b0 + lane;
             const int j = u0 + u;
-            const AT cn_a = fma(vf, (AT)c_s[u * B + b], vi * vg);
+            const GT cn_a = fma(vf, (GT)c_s[u * B + b], vi * vg);
             const float cn = (float)cn_a;
             const float hn = (float)(vo * tanh_t(cn_a));
             if ((int)blockIdx.x != a.withhold_cta)
