@@ -106,14 +106,12 @@ __device__ __forceinline__ void unit_dot_dense(const WT *rows, int Hp8, const fl
             load_w8(rows + (size_t)q * Hp8, v8, w);
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
-                // eight terms in fp32 (two chains of four; their rounding error is a few 1e-8 of the terms'
-                // size), the partial sums added up in AT: with a double or two-float AT the long sum over H
-                // stays exact to far below fp32 rounding
-                float s0 = w[0] * hlo[b].x, s1 = w[4] * hhi[b].x;
-                s0 = fmaf(w[1], hlo[b].y, s0); s1 = fmaf(w[5], hhi[b].y, s1);
-                s0 = fmaf(w[2], hlo[b].z, s0); s1 = fmaf(w[6], hhi[b].z, s1);
-                s0 = fmaf(w[3], hlo[b].w, s0); s1 = fmaf(w[7], hhi[b].w, s1);
-                acc[q * BT + b] += (AT)(s0 + s1);
+                AT s = acc[q * BT + b];
+                s = fma((AT)w[0], (AT)hlo[b].x, s); s = fma((AT)w[1], (AT)hlo[b].y, s);
+                s = fma((AT)w[2], (AT)hlo[b].z, s); s = fma((AT)w[3], (AT)hlo[b].w, s);
+                s = fma((AT)w[4], (AT)hhi[b].x, s); s = fma((AT)w[5], (AT)hhi[b].y, s);
+                s = fma((AT)w[6], (AT)hhi[b].z, s); s = fma((AT)w[7], (AT)hhi[b].w, s);
+                acc[q * BT + b] = s;
             }
         }
     }
@@ -150,20 +148,21 @@ __device__ __forceinline__ void unit_dot_csr(const ET *ent, const int (&e)[5], c
         decode4(ent, vi, w, col);
 #pragma unroll
         for (int b = 0; b < BT; ++b) {
-            float s = w[0] * hb[b * Hs + col[0]];
-            s = fmaf(w[1], hb[b * Hs + col[1]], s);
-            s = fmaf(w[2], hb[b * Hs + col[2]], s);
-            s = fmaf(w[3], hb[b * Hs + col[3]], s);
+            AT s = (AT)w[0] * (AT)hb[b * Hs + col[0]];
+            s = fma((AT)w[1], (AT)hb[b * Hs + col[1]], s);
+            s = fma((AT)w[2], (AT)hb[b * Hs + col[2]], s);
+            s = fma((AT)w[3], (AT)hb[b * Hs + col[3]], s);
 #pragma unroll
-            for (int qq = 0; qq < 4; ++qq) acc[qq * BT + b] += (AT)((q == qq) ? s : 0.0f);
+            for (int qq = 0; qq < 4; ++qq) acc[qq * BT + b] += (q == qq) ? s : (AT)0;
         }
     }
 }
 
-// bf16 storage: fp32 accumulation and gate functions.  fp32 storage: short fp32 chains of four or eight terms
-// added up in fp64, and the gate functions and the state update in fp64, so the only fp32 roundings left are
-// the stored projection, h and c -- what the 1e-4 agreement bound of that mode needs (two-float sums with fp32
-// gate functions were measured: 1.02e-4 on the floored metric, and no faster: the step waits for the exchange).
+// bf16 storage: fp32 accumulation and gate functions.  fp32 storage: dot products accumulate in fp64
+// and the gate functions are evaluated in fp64, so the only fp32 roundings left are the stored
+// projection, h and c -- what the 1e-4 agreement bound of that mode needs.  Cheaper forms were measured
+// and miss it: fp32 chains of eight terms summed in fp64 (1.2e-4 on the floored metric at H = 300, B = 16),
+// two-float sums with fp32 gate functions (1.02e-4); neither shortened the step, which waits for the exchange.
 template <bool BF16> struct Types { typedef __nv_bfloat16 W; typedef unsigned E; typedef float A; };
 template <> struct Types<false> { typedef float W; typedef CsrEntry E; typedef double A; };
 
