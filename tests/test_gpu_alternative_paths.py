@@ -1,0 +1,90 @@
+"""The code paths the environment switches select instead of the defaults must stay correct: they are what the
+defaults are measured against (issuing threads of the batched recurrence, 128-row projection tiles, the
+list-walking projection of CSR handles), and some are the only path for shapes the default does not serve."""
+import numpy as np
+import pytest
+
+import lstm_workloads as wl
+from gpu_util import assert_close, csr_weights
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, layers, bidir, in_dim, hidden, T, B, dtype, scale=0.1, seed=7, density=1.0):
+    return wl.Workload(name, layers, bidir, in_dim, hidden, T, B, dtype, scale, density=density, seed=seed)
+
+
+def _forward(pkg, w, weights, x, h0, c0, exec_mode="dense"):
+    import torch
+    m = pkg.LSTM(weights, layers=w.layers, in_dim=w.in_dim, hidden=w.hidden, bidir=w.bidir, dtype=w.dtype,
+                 exec_mode=exec_mode, max_T=w.T, max_B=w.B)
+    try:
+        y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
+        m.check()
+        return (y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), m.info()
+    finally:
+        m.close()
+
+
+@pytest.mark.parametrize("issuers", ["1", "2"])
+def test_batched_recurrence_with_fewer_issuing_threads(oracle, issuers, monkeypatch):
+    """One and two issuing threads (one and two accumulators) instead of three; pair mode and both directions,
+    and a slice whose ring does not hold a whole step's operand."""
+    import paper_1901_10997_b200 as pkg
+    monkeypatch.setenv("LSTM_B200_TC_ISSUE", issuers)
+    for w in (small("tci_h600_b20", 1, True, 24, 600, 3, 20, "bf16", scale=0.05),
+              small("tci_h1600_b9", 1, False, 32, 1600, 2, 9, "bf16", scale=0.03)):
+        weights, x = wl.make(w)
+        h0, c0 = wl.make_states(w)
+        ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        got, info = _forward(pkg, w, weights, x, h0, c0)
+        assert info["recur_batched_tensor_core"] >= 1
+        assert_close(got, ref, "bf16", f"{w.name}/issuers={issuers}")
+
+
+def test_batched_recurrence_without_cluster_pairs(oracle, monkeypatch):
+    import paper_1901_10997_b200 as pkg
+    monkeypatch.setenv("LSTM_B200_RECUR", "tc1")
+    w = small("tc1_h600_b20", 2, False, 24, 600, 3, 20, "bf16", scale=0.05)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got, info = _forward(pkg, w, weights, x, h0, c0)
+    assert info["recur_batched_tensor_core"] == 1
+    assert_close(got, ref, "bf16", w.name)
+
+
+@pytest.mark.parametrize("tile", ["128", ""])
+def test_projection_tiles_at_several_activation_tiles(oracle, tile, monkeypatch):
+    """T*B = 390 rows (four activation tiles, a ragged last one) and 4H = 1160 weight rows (a ragged 256-row tile):
+    the persistent 256-row kernel (default) and the 128-row kernel, through the whole forward pass."""
+    import paper_1901_10997_b200 as pkg
+    if tile:
+        monkeypatch.setenv("LSTM_B200_PROJ_TILE", tile)
+    else:
+        monkeypatch.delenv("LSTM_B200_PROJ_TILE", raising=False)
+    w = small("proj_tiles", 2, False, 200, 290, 13, 30, "bf16", scale=0.05)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got, _ = _forward(pkg, w, weights, x, h0, c0)
+    assert_close(got, ref, "bf16", f"{w.name}/tile={tile or 'default'}")
+
+
+@pytest.mark.parametrize("proj", ["csr", ""])
+def test_csr_handle_with_either_projection(oracle, proj, monkeypatch):
+    """bf16 CSR handles project on the tensor cores over a dense copy of Wx by default and walk the lists with
+    LSTM_B200_PROJ=csr; two layers, so that the second projection reads what the sparse recurrence wrote."""
+    import paper_1901_10997_b200 as pkg
+    if proj:
+        monkeypatch.setenv("LSTM_B200_PROJ", proj)
+    else:
+        monkeypatch.delenv("LSTM_B200_PROJ", raising=False)
+    for B in (1, 3):
+        w = small("csr_proj", 2, True, 70, 200, 6, B, "bf16", scale=0.2, density=0.15, seed=5)
+        weights, x = wl.make(w)
+        h0, c0 = wl.make_states(w)
+        ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+        got, info = _forward(pkg, w, csr_weights(oracle, weights), x, h0, c0, exec_mode="csr")
+        assert info["proj_tensor_core"] == (0 if proj else 1)
+        assert_close(got, ref, "bf16", f"{w.name}/B={B}/proj={proj or 'default'}")
