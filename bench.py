@@ -771,7 +771,18 @@ def run_matmul_sweep(args):
             w = wl.Workload(f"matmul_d{dsz}", 1, False, dsz, H, 16, 1, "bf16", 1.0 / np.sqrt(dsz), density=density,
                             seed=wl.SEED_BASE + dsz)
             weights, x = wl.make(w)
-            m = pkg.LSTM(weights, layers=1, in_dim=dsz, hidden=H, dtype="bf16", exec_mode=mode, max_T=16, max_B=1)
+            # the sparse arms walk the lists (by default a bf16 CSR handle would project on the tensor cores over a
+            # dense copy of the matrix, which is the dense arm again)
+            old_env = os.environ.get("LSTM_B200_PROJ")
+            if mode == "csr":
+                os.environ["LSTM_B200_PROJ"] = "csr"
+            try:
+                m = pkg.LSTM(weights, layers=1, in_dim=dsz, hidden=H, dtype="bf16", exec_mode=mode, max_T=16, max_B=1)
+            finally:
+                if old_env is None:
+                    os.environ.pop("LSTM_B200_PROJ", None)
+                else:
+                    os.environ["LSTM_B200_PROJ"] = old_env
             xd = torch.from_numpy(x).to(dev)
             out = torch.empty((16, 1, 1, 4 * H), device=dev)
             fn = lambda: m.input_projection(xd, out=out)
