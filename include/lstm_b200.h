@@ -142,7 +142,7 @@ LSTM_API int lstm_create(lstm_handle **out, int layers, int in_dim, int hidden, 
  * followed by the same gate functions and c/h update as above.  Weights of one (layer, direction), all
  * row-major fp32, host or device pointers, read only during the call:
  *   ux [4Hh, in_l], uh [4Hh, H]: rows q*Hh + m;  a [4Hh] or NULL;  w [4H, Hh]: row q*H + j multiplies r_q;
- *   b [4H] or NULL.  A pruned weight is passed as an explicit zero (W (x) Msk).
+ *   b [4H] or NULL.  Pruned weights: explicit zeros in ux, uh, w, or the keep-masks below.
  * hlstm_create returns a handle that lstm_forward, lstm_forward_host, lstm_status, lstm_destroy and the
  * other calls accept like an LSTM handle.  Only LSTM_BF16W_F32S storage is served; sizes whose per-CTA
  * slices of Uh and W do not fit registers + shared memory (roughly hidden, gate_hidden > 1700) return
@@ -154,6 +154,11 @@ typedef struct {
     const float *a;
     const float *w;
     const float *b;
+    /* optional keep-masks (Section 4.2: W (x) Msk), one byte per weight, non-zero = kept, same shapes as ux, uh
+     * and w; NULL keeps every weight.  A masked weight is multiplied as an explicit zero. */
+    const unsigned char *mask_ux;
+    const unsigned char *mask_uh;
+    const unsigned char *mask_w;
 } hlstm_weights;
 
 LSTM_API int hlstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int gate_hidden, int bidir, int dtype,

@@ -38,7 +38,7 @@ class _Weights(ctypes.Structure):
 
 
 class _HWeights(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("ux", "uh", "a", "w", "b")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("ux", "uh", "a", "w", "b", "mask_ux", "mask_uh", "mask_w")]
 
 
 def lib_path() -> Path:
@@ -394,7 +394,8 @@ class LSTM:
 
 class HLSTM(LSTM):
     """H-LSTM cell (one ReLU hidden layer of width ``gate_hidden`` inside each gate).  ``weights``: list of
-    dicts per (layer, direction) with ``ux`` [4Hh,in_l], ``uh`` [4Hh,H], ``w`` [4H,Hh], optional ``a``, ``b``;
+    dicts per (layer, direction) with ``ux`` [4Hh,in_l], ``uh`` [4Hh,H], ``w`` [4H,Hh], optional ``a``, ``b`` and
+    keep-masks ``mask_ux``, ``mask_uh``, ``mask_w`` (uint8, same shapes);
     gate blocks i, f, g, o.  Forward, status and the other methods are those of ``LSTM``."""
 
     def __init__(self, weights, *, layers, in_dim, hidden, gate_hidden, bidir=False, dtype="bf16", max_T, max_B, stream=0):
@@ -415,6 +416,8 @@ class HLSTM(LSTM):
             s.w = _addr(_as_c(w["w"], np.float32), keep)
             s.a = _addr(_as_c(w.get("a"), np.float32), keep)
             s.b = _addr(_as_c(w.get("b"), np.float32), keep)
+            for name in ("mask_ux", "mask_uh", "mask_w"):
+                setattr(s, name, _addr(_as_c(w.get(name), np.uint8), keep))
         dt = {"fp32": LSTM_F32, "bf16": LSTM_BF16W_F32S}[dtype]
         rc, handle = hlstm_create(self.layers, self.in_dim, self.hidden, self.gate_hidden, bidir, dt,
                                   ctypes.cast(arr, ctypes.c_void_p), self.max_T, self.max_B, stream)

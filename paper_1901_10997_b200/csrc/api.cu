@@ -1071,6 +1071,20 @@ int hlstm_create(lstm_handle **out, int layers, int in_dim, int hidden, int gate
                 !host_view(src.b, sizeof(float) * 4 * H, v_b)) { rc = fail(h, LSTM_ERR_CUDA, "reading weights"); break; }
             const float *ux = (const float *)v_ux.ptr, *uh = (const float *)v_uh.ptr, *ww = (const float *)v_w.ptr;
             const float *ba = (const float *)v_a.ptr, *bb = (const float *)v_b.ptr;
+            // keep-masks: the masked copies replace the caller's matrices
+            std::vector<float> ux_m, uh_m, w_m;
+            auto masked = [&](const float *&m, const unsigned char *mask, size_t n, std::vector<float> &store) -> bool {
+                if (!mask) return true;
+                HostView v;
+                if (!host_view(mask, n, v)) return false;
+                const unsigned char *mk = (const unsigned char *)v.ptr;
+                store.resize(n);
+                for (size_t i = 0; i < n; ++i) store[i] = mk[i] ? m[i] : 0.0f;
+                m = store.data();
+                return true;
+            };
+            if (!masked(ux, src.mask_ux, (size_t)4 * Hh * ly.in_l, ux_m) || !masked(uh, src.mask_uh, (size_t)4 * Hh * H, uh_m) ||
+                !masked(ww, src.mask_w, (size_t)4 * H * Hh, w_m)) { rc = fail(h, LSTM_ERR_CUDA, "reading masks"); break; }
             for (int q = 0; q < 4; ++q) {
                 for (int m = 0; m < Hh; ++m) {
                     const size_t prow = (size_t)d * 4 * Hh + (size_t)m * 4 + q;           // unit-major, gates adjacent

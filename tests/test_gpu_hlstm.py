@@ -106,3 +106,23 @@ def test_hlstm_random_shapes(oracle, c):
     h0, c0 = wl.make_states(w)
     ref = oracle.forward_hlstm(weights, x, h0, c0, layers=c["L"], bidir=c["bidir"], hidden=c["H"], gate_hidden=c["Hh"])
     assert_close(run(w, c["Hh"], weights, x, h0, c0), ref, "bf16", "hlstm fuzz")
+
+
+def test_hlstm_keep_masks_equal_explicit_zeros(oracle):
+    """Pruned H-LSTM (the model the paper ships, Table 1 row (d)): keep-masks given to the library against the
+    oracle run on W (x) Msk written out; 80 % of every matrix pruned, two layers, both directions."""
+    L, bidir, in_dim, H, Hh, T, B = 2, True, 24, 150, 130, 5, 2
+    w = wl.Workload("hlstm_masked", L, bidir, in_dim, H, T, B, "bf16", 0.5, seed=77)
+    weights, x = wl.make_hlstm(w, Hh)
+    h0, c0 = wl.make_states(w)
+    rng = np.random.default_rng(123)
+    masked, zeroed = [], []
+    for ws in weights:
+        m = {k: (rng.random(ws[k].shape) < 0.2).astype(np.uint8) for k in ("ux", "uh", "w")}
+        masked.append(dict(ws, mask_ux=m["ux"], mask_uh=m["uh"], mask_w=m["w"]))
+        zeroed.append(dict(ws, ux=ws["ux"] * m["ux"], uh=ws["uh"] * m["uh"], w=ws["w"] * m["w"]))
+    ref = oracle.forward_hlstm(zeroed, x, h0, c0, layers=L, bidir=bidir, hidden=H, gate_hidden=Hh)
+    got = run(w, Hh, masked, x, h0, c0)
+    assert_close(got, ref, "bf16", "hlstm/masks")
+    dense_ref = oracle.forward_hlstm(weights, x, h0, c0, layers=L, bidir=bidir, hidden=H, gate_hidden=Hh)
+    assert np.abs(dense_ref[0] - ref[0]).max() > 1e-2          # the masks change the result: they were applied
