@@ -60,6 +60,7 @@ struct lstm_handle {
     bool fuse_ok = false;              // short single sequences: projection fused into the register-resident kernel's prologue
     // register-resident sparse kernel (bf16, CSR execution): warps, columns per warp, row tiles, entry slots per lane
     bool use_csr_reg = false;
+    bool csr_fuse_ok = false;          // register-resident sparse kernel: single short sequences project in its prologue
     bool csr_dense_proj = false;       // CSR handle whose input projection runs on the tensor cores over Wx with explicit zeros
     int csr_nw = 0, csr_kspan = 0, csr_mt = 0, csr_slots = 0;
     long long csr_conflicts = 0;       // shared-memory wavefronts per step and CTA lost to bank conflicts (worst CTA, worst matrix)
@@ -553,6 +554,9 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         if (!(env && strcmp(env, "simt") == 0) && h->upc <= nw &&
             recur_csr_reg_smem_bytes(nw, kspan, mt, h->upc, max_B) <= (size_t)h->smem_optin - 64) {
             h->use_csr_reg = true; h->csr_nw = nw; h->csr_kspan = kspan; h->csr_mt = mt;
+            const char *fenv = getenv("LSTM_B200_FUSE");
+            h->csr_fuse_ok = h->csr_dense_proj && nw == 16 && mt <= 4 && !(fenv && strcmp(fenv, "0") == 0) &&
+                             recur_csr_reg_fuse_smem_bytes(nw, kspan, mt, h->upc) <= (size_t)h->smem_optin - 64;
         }
     }
     // does the batched tensor-core recurrence fit with the current split of the SMs?
@@ -727,6 +731,19 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                         }
                         px_rowptr[(size_t)d * 4 * H + (size_t)j * 4 + q + 1] = (int)px_ent.size();
                     }
+                if (h->csr_fuse_ok) {
+                    // Wx with its zeros as operand-A fragments: single short sequences project in the sparse
+                    // recurrent kernel's prologue, on the tensor cores (two warps share a column range)
+                    std::vector<float> m((size_t)4 * H * ly.in_l, 0.0f);
+                    for (int r = 0; r < 4 * H; ++r)
+                        for (int e = cx.rowptr[r]; e < cx.rowptr[r + 1]; ++e) m[(size_t)r * ly.in_l + cx.col[e]] = cx.val[e];
+                    const int nranges = h->csr_nw / 2;
+                    ly.nkw_x = ((ly.in_l + 15) / 16 + nranges - 1) / nranges;
+                    const std::vector<uint32_t> fx = pack_fragments(m.data(), H, ly.in_l, h->ncta_dir, nranges, ly.nkw_x, h->csr_mt);
+                    rc = upload(h, (uint32_t **)&ly.xfrag[d], fx.data(), fx.size() * 4, st, "input weight fragments");
+                    if (rc == LSTM_OK) cudaStreamSynchronize(st);
+                    if (rc) break;
+                }
                 snprintf(name, sizeof name, "wh[layer %d, dir %d]", l, d);
                 rc = matrix_to_csr(h, 4 * H, H, src.wh, src.mask_h, src.wh_rowptr, src.wh_col, src.wh_val, ch, name);
                 if (rc) break;
@@ -784,6 +801,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
         // one slot count for the whole handle: the longest lane list of any matrix, rounded up to a built size
         const int slots = recur_csr_reg_slots(std::max(h->csr_slots, 1), h->csr_nw);
         if (slots == 0) h->use_csr_reg = false;            // lists too long for registers: the shared-memory kernel runs
+        if (!h->use_csr_reg) h->csr_fuse_ok = false;
         h->csr_slots = slots;
         for (int l = 0; l < layers && rc == LSTM_OK; ++l)
             for (int d = 0; d < D && rc == LSTM_OK; ++d) {
@@ -1298,7 +1316,8 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
         int nsplit = 1;
         // ---- input staging + projection (a single short sequence on the register-resident kernel computes its
         // projection inside that kernel's prologue instead: two launches and one round trip of G fewer per layer)
-        const bool fuse = h->fuse_ok && !h->Hh && B == 1 && T <= kFuseMaxT && !h->probe && ly.xfrag[0] != nullptr;
+        const bool fuse = (h->fuse_ok || (h->csr_fuse_ok && h->use_csr_reg)) && !h->Hh && B == 1 && T <= kFuseMaxT && !h->probe &&
+                          ly.xfrag[0] != nullptr;
         if (!fuse) { const int prc = run_projection(h, l, l == 0 ? x : nullptr, Xf, M, N, &nsplit, st); if (prc != LSTM_OK) return prc; }
 
         // ---- recurrence: all directions in one launch, or one launch per direction
@@ -1407,12 +1426,17 @@ int lstm_forward(lstm_handle *h, const float *x, int T, int B, const float *h0, 
             m.h0 = h0 ? h0 + so : nullptr; m.c0 = c0 ? c0 + so : nullptr;
             m.hT = hT ? hT + so : nullptr; m.cT = cT ? cT + so : nullptr;
             m.y = l == L - 1 ? y : h->ybuf[l & 1];
-            m.xb_next = (l < L - 1 && h->use_tc) ? h->xbn[l & 1] : nullptr;
+            m.xb_next = (l < L - 1 && h->use_tc && !fuse) ? h->xbn[l & 1] : nullptr;     // a fused next layer reads the fp32 activations
             m.xb_ld = h->ldn;
             m.xb_plane = (long long)h->max_T * h->max_B * h->ldn;
             m.xch = h->xch;
             m.status = h->status_dev;
-            const size_t smem = recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, B);
+            m.fuse = fuse ? 1 : 0;
+            m.in_l = ly.in_l; m.nkw_x = ly.nkw_x; m.X = Xf; m.bias = ly.bias;
+            m.gs_off = (int)recur_csr_reg_fuse_gs_offset(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc);
+            for (int d = 0; d < D; ++d) m.xfrag[d] = ly.xfrag[d];
+            const size_t smem = fuse ? recur_csr_reg_fuse_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc)
+                                     : recur_csr_reg_smem_bytes(h->csr_nw, h->csr_kspan, h->csr_mt, h->upc, B);
             if (record(h, LSTM_K_RECUR, st)) return fail(h, LSTM_ERR_CUDA, "event record failed");
             e = launch_recur_csr_reg(m, h->csr_slots, h->csr_nw, smem, st);
             ++h->last_launches;

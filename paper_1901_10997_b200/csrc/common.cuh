@@ -170,7 +170,14 @@ struct RecurCsrArgs {
     int xb_ld;
     unsigned long long *xch;
     int *status;
+    // projection fused into the prologue (single sequence, T <= kFuseMaxT): Wx as operand-A fragments of a dense
+    // copy (zeros included), layout as in RecurMmaArgs with NW / 2 column ranges
+    int fuse, in_l, nkw_x, gs_off;
+    const float *X, *bias;
+    const uint4 *xfrag[2];
 };
+size_t recur_csr_reg_fuse_gs_offset(int nw, int kspan, int mt, int upc);
+size_t recur_csr_reg_fuse_smem_bytes(int nw, int kspan, int mt, int upc);
 constexpr int kCsrRegMaxSlots16 = 64;    // entry slots per lane the kernel is built for with 16 warps ...
 constexpr int kCsrRegMaxSlots8 = 128;    // ... and with 8 warps (255 registers per thread)
 int recur_csr_reg_slots(int needed, int nw);     // smallest built slot count >= needed, or 0 when none is

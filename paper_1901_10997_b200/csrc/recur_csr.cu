@@ -22,14 +22,18 @@
 #include "device_util.cuh"
 #include "recur_parts.cuh"
 
+#include <algorithm>
+
 namespace lstm {
 namespace {
 
 constexpr int kChunk = 4;      // batch rows per pass
 constexpr int kMaxSplit = 4;   // split-K planes of the projection output
 
-// E: entry slots per lane; NW: warps per CTA; ONE: a single sequence (B = 1); PROBE: measurement build.
-template <int E, int NW, bool ONE, bool PROBE>
+// E: entry slots per lane; NW: warps per CTA; ONE: a single sequence (B = 1); PROBE: measurement build;
+// FUSE: the CTA computes its own rows of the layer's input projection in the prologue (single short sequence),
+// on the tensor cores over a dense copy of Wx, and reads the projection terms from shared memory afterwards.
+template <int E, int NW, bool ONE, bool PROBE, bool FUSE = false>
 __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArgs a)
 {
     constexpr int NT = NW * 32;
@@ -56,6 +60,20 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArg
     float *red = hs + (size_t)NW * hstride;                      // [2][NW][WS]
     float *c_s = red + 2 * NW * WS;                              // [upc][B]
     LSTM_CHECK_SMEM_END((size_t)(reinterpret_cast<unsigned char *>(c_s + ((upc * B + 3) & ~3)) - smem), a.status);
+
+    // ---- the CTA's rows of the input projection (before anything else lives in shared memory or registers)
+    const float *G_s = nullptr;
+    const int GP = a.mt * 16 + 1;
+    if (FUSE) {
+        LSTM_CHECK_SMEM_END((size_t)a.gs_off + (size_t)kFuseMaxT * GP * 4, a.status);
+        LSTM_CHECK_SMEM_END((size_t)NW * 24 * GP * 4, a.status);
+        switch (a.mt) {
+            case 1: G_s = fused_projection<1, NW>(smem, (size_t)a.gs_off, a.X, a.xfrag[d], a.bias, a.nkw_x, a.in_l, T, H, d, cta, u0, nu, tid); break;
+            case 2: G_s = fused_projection<2, NW>(smem, (size_t)a.gs_off, a.X, a.xfrag[d], a.bias, a.nkw_x, a.in_l, T, H, d, cta, u0, nu, tid); break;
+            case 3: G_s = fused_projection<3, NW>(smem, (size_t)a.gs_off, a.X, a.xfrag[d], a.bias, a.nkw_x, a.in_l, T, H, d, cta, u0, nu, tid); break;
+            default: G_s = fused_projection<4, NW>(smem, (size_t)a.gs_off, a.X, a.xfrag[d], a.bias, a.nkw_x, a.in_l, T, H, d, cta, u0, nu, tid); break;
+        }
+    }
 
     // ---- residency: this lane's entry list and its rows
     unsigned ent[E];
@@ -103,7 +121,9 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArg
             float gv[kMaxSplit];
 #pragma unroll
             for (int sp = 0; sp < kMaxSplit; ++sp) gv[sp] = 0.0f;
-            if (fin_warp && f.fpart == 0 && b0 + f.fb < B) {
+            if (FUSE) {
+                if (fin_warp && f.fpart == 0) gv[0] = G_s[(size_t)t * GP + warp * 4 + f.fq];
+            } else if (fin_warp && f.fpart == 0 && b0 + f.fb < B) {
                 const float *gp = a.G + (((size_t)t * B + b0 + f.fb) * D + d) * 4 * H + (size_t)(u0 + warp) * 4 + f.fq;
 #pragma unroll
                 for (int sp = 0; sp < kMaxSplit; ++sp)
@@ -192,19 +212,19 @@ __global__ void __launch_bounds__(NW * 32, 1) recur_csr_kernel(const RecurCsrArg
 
 typedef void (*KernelFn)(const RecurCsrArgs);
 
-template <int NW, bool ONE, bool PROBE>
+template <int NW, bool ONE, bool PROBE, bool FUSE = false>
 KernelFn pick_slots(int slots)
 {
     switch (slots) {
-        case 8: return recur_csr_kernel<8, NW, ONE, PROBE>;
-        case 16: return recur_csr_kernel<16, NW, ONE, PROBE>;
-        case 20: return recur_csr_kernel<20, NW, ONE, PROBE>;
-        case 24: return recur_csr_kernel<24, NW, ONE, PROBE>;
-        case 28: return recur_csr_kernel<28, NW, ONE, PROBE>;
-        case 32: return recur_csr_kernel<32, NW, ONE, PROBE>;
-        case 40: return recur_csr_kernel<40, NW, ONE, PROBE>;
-        case 48: return recur_csr_kernel<48, NW, ONE, PROBE>;
-        case 64: return recur_csr_kernel<64, NW, ONE, PROBE>;
+        case 8: return recur_csr_kernel<8, NW, ONE, PROBE, FUSE>;
+        case 16: return recur_csr_kernel<16, NW, ONE, PROBE, FUSE>;
+        case 20: return recur_csr_kernel<20, NW, ONE, PROBE, FUSE>;
+        case 24: return recur_csr_kernel<24, NW, ONE, PROBE, FUSE>;
+        case 28: return recur_csr_kernel<28, NW, ONE, PROBE, FUSE>;
+        case 32: return recur_csr_kernel<32, NW, ONE, PROBE, FUSE>;
+        case 40: return recur_csr_kernel<40, NW, ONE, PROBE, FUSE>;
+        case 48: return recur_csr_kernel<48, NW, ONE, PROBE, FUSE>;
+        case 64: return recur_csr_kernel<64, NW, ONE, PROBE, FUSE>;
         default: return nullptr;
     }
 }
@@ -219,11 +239,13 @@ KernelFn pick_nw(int slots, int nw)
     }
     return nullptr;
 }
-// variant 0: up to four sequences per pass, 1: one sequence, 2: the measurement build of 1
+// variant 0: up to four sequences per pass, 1: one sequence, 2: the measurement build of 1, 3: one sequence with
+// the projection in the prologue (16 warps only)
 KernelFn pick(int slots, int nw, int variant)
 {
     if (variant == 0) return pick_nw<false, false>(slots, nw);
     if (variant == 1) return pick_nw<true, false>(slots, nw);
+    if (variant == 3) return nw == 16 ? pick_slots<16, true, false, true>(slots) : nullptr;
     return pick_nw<true, true>(slots, nw);
 }
 
@@ -251,10 +273,24 @@ size_t recur_csr_reg_smem_bytes(int nw, int kspan, int mt, int upc, int B)
     return ((size_t)nw * recur_csr_reg_hs_stride(kspan, B) + (size_t)2 * nw * red_warp_pitch(mt) + (size_t)((upc * B + 3) & ~3)) * 4;
 }
 
+// fused projection: the partial products of all warps (24 timesteps x rows each) lie over the kernel's other
+// shared memory, the finished rows of G behind whichever is larger
+size_t recur_csr_reg_fuse_gs_offset(int nw, int kspan, int mt, int upc)
+{
+    const size_t normal = recur_csr_reg_smem_bytes(nw, kspan, mt, upc, 1);
+    const size_t partial = (size_t)nw * 24 * (mt * 16 + 1) * 4;
+    return (std::max(normal, partial) + 15) & ~(size_t)15;
+}
+size_t recur_csr_reg_fuse_smem_bytes(int nw, int kspan, int mt, int upc)
+{
+    return recur_csr_reg_fuse_gs_offset(nw, kspan, mt, upc) + (size_t)kFuseMaxT * (mt * 16 + 1) * 4;
+}
+
 cudaError_t recur_csr_reg_prepare(int slots, int nw, int max_smem)
 {
-    for (int variant = 0; variant < 3; ++variant) {
+    for (int variant = 0; variant < 4; ++variant) {
         KernelFn fn = pick(slots, nw, variant);
+        if (!fn && variant == 3) continue;                      // no fused build for this warp count
         if (!fn) return cudaErrorInvalidValue;
         const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
         if (e != cudaSuccess) return e;
@@ -265,6 +301,10 @@ cudaError_t recur_csr_reg_prepare(int slots, int nw, int max_smem)
 cudaError_t launch_recur_csr_reg(const RecurCsrArgs &a, int slots, int nw, size_t smem, cudaStream_t st)
 {
     int variant = a.B == 1 ? 1 : 0;
+    if (a.fuse) {
+        if (a.B != 1 || a.probe || nw != 16 || a.T > kFuseMaxT) return cudaErrorInvalidValue;
+        variant = 3;
+    }
     if (a.probe) {
         if (variant != 1) return cudaErrorInvalidValue;
         variant = 2;

@@ -126,4 +126,105 @@ __device__ __forceinline__ void finish_unit(const FinishLane &f, const float *re
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------
+// Input projection inside a recurrent kernel's prologue (single sequence of at most kFuseMaxT steps): the CTA's
+// own rows of G = X Wx^T + b for every timestep, left in shared memory as [kFuseMaxT][MT * 16 + 1] floats at
+// byte offset gs_off.  Wx arrives as mma.sync operand-A fragments (xfrag_d: this direction's, laid out
+// [cta][NW / 2 column ranges][nkx 16-column tiles][MT][32 lanes] uint4); the activations are split into bf16 hi
+// and lo terms on the fly.  Work split: the NW / 2 column ranges are each taken by two warps, one for the first
+// 24 timesteps and one for the rest, so that the accumulators of a warp stay few and two loads can be in flight.
+// Every warp leaves its partial products in its own block at the start of shared memory (NW * 24 * (MT * 16 + 1)
+// floats, over memory the caller initialises only afterwards); then each (timestep, row) adds its NW / 2 partial
+// sums in a fixed order and the bias.  All NW * 32 threads of the CTA call it; it ends with a CTA barrier.
+template <int MT, int NW>
+__device__ __forceinline__ float *fused_projection(unsigned char *smem, size_t gs_off, const float *X, const uint4 *xfrag_d,
+                                                   const float *bias, int nkx, int in_l, int T, int H, int d, int cta,
+                                                   int u0, int nu, int tid)
+{
+    constexpr int NT = NW * 32, NR = NW / 2, NTH = 3, GP = MT * 16 + 1;     // column ranges; 8-step tiles per warp
+    const int lane = tid & 31, warp = tid >> 5, g = lane >> 2, tig = lane & 3;
+    const int range = warp >> 1, half = warp & 1;
+    const uint4 *xbase = xfrag_d + ((size_t)(cta * NR + range) * nkx) * MT * 32;
+    for (int i = lane + 32 * half; i < nkx * MT * 4; i += 64)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xbase) + (size_t)i * 128));
+    float *G_s = nullptr;
+    float pacc[MT][NTH][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTH; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) pacc[mt][nt][e] = 0.0f;
+    const uint4 *xsrc = xbase + lane;
+    const int t0 = half * NTH * 8;
+    uint4 af[MT], an[MT];
+    float xv[NTH][4], xn[NTH][4];
+    auto fetch = [&](int i, uint4 (&fa)[MT], float (&fx)[NTH][4]) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) fa[mt] = i < nkx ? __ldg(xsrc + (size_t)(i * MT + mt) * 32) : make_uint4(0, 0, 0, 0);
+        const int k0 = (range * nkx + i) * 16 + 2 * tig;
+#pragma unroll
+        for (int nt = 0; nt < NTH; ++nt) {
+            const int t = t0 + nt * 8 + g;
+            const float *xr = X + (size_t)t * in_l;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int k = k0 + (e & 1) + (e >> 1) * 8;
+                fx[nt][e] = (i < nkx && t < T && k < in_l) ? __ldg(xr + k) : 0.0f;
+            }
+        }
+    };
+    fetch(0, af, xv);
+#pragma unroll 1
+    for (int i = 0; i < nkx; ++i) {
+        fetch(i + 1, an, xn);
+#pragma unroll
+        for (int nt = 0; nt < NTH; ++nt) {
+            const __nv_bfloat162 h01 = __floats2bfloat162_rn(xv[nt][0], xv[nt][1]), h23 = __floats2bfloat162_rn(xv[nt][2], xv[nt][3]);
+            const __nv_bfloat162 l01 = __floats2bfloat162_rn(xv[nt][0] - __low2float(h01), xv[nt][1] - __high2float(h01));
+            const __nv_bfloat162 l23 = __floats2bfloat162_rn(xv[nt][2] - __low2float(h23), xv[nt][3] - __high2float(h23));
+            const unsigned bh0 = *reinterpret_cast<const unsigned *>(&h01), bh1 = *reinterpret_cast<const unsigned *>(&h23);
+            const unsigned bl0 = *reinterpret_cast<const unsigned *>(&l01), bl1 = *reinterpret_cast<const unsigned *>(&l23);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                mma_bf16(pacc[mt][nt], af[mt], bh0, bh1);
+                mma_bf16(pacc[mt][nt], af[mt], bl0, bl1);
+            }
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) af[mt] = an[mt];
+#pragma unroll
+        for (int nt = 0; nt < NTH; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) xv[nt][e] = xn[nt][e];
+    }
+    // every warp leaves its partial products in its own block (the blocks lie over shared memory that is only
+    // initialised afterwards); then each (timestep, row) adds its NR partial sums in a fixed order and the bias
+    constexpr int PP = MT * 16 + 1;
+    float *P = reinterpret_cast<float *>(smem) + (size_t)warp * (NTH * 8) * PP;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTH; ++nt) {
+            float *pp = P + (size_t)(nt * 8 + 2 * tig) * PP + mt * 16 + g;
+            pp[0] = pacc[mt][nt][0];
+            pp[PP] = pacc[mt][nt][1];
+            pp[8] = pacc[mt][nt][2];
+            pp[PP + 8] = pacc[mt][nt][3];
+        }
+    __syncthreads();
+    G_s = reinterpret_cast<float *>(smem + gs_off);
+    for (int i = tid; i < kFuseMaxT * MT * 16; i += NT) {
+        const int t = i / (MT * 16), r = i - t * (MT * 16);
+        const int hf = t / (NTH * 8), tl = t - hf * (NTH * 8);
+        float sum = r < 4 * nu ? bias[(size_t)d * 4 * H + (size_t)u0 * 4 + r] : 0.0f;
+#pragma unroll
+        for (int rg = 0; rg < NR; ++rg) sum += reinterpret_cast<const float *>(smem)[((size_t)(2 * rg + hf) * (NTH * 8) + tl) * PP + r];
+        G_s[(size_t)t * GP + r] = sum;
+    }
+    __syncthreads();
+    return G_s;
+}
+
 }  // namespace lstm

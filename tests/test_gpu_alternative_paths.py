@@ -88,3 +88,28 @@ def test_csr_handle_with_either_projection(oracle, proj, monkeypatch):
         got, info = _forward(pkg, w, csr_weights(oracle, weights), x, h0, c0, exec_mode="csr")
         assert info["proj_tensor_core"] == (0 if proj else 1)
         assert_close(got, ref, "bf16", f"{w.name}/B={B}/proj={proj or 'default'}")
+
+
+@pytest.mark.parametrize("T,fused", [(37, True), (41, False)])
+def test_sparse_kernel_projects_in_its_prologue_for_short_single_sequences(oracle, T, fused, monkeypatch):
+    """bf16 CSR handle on the 16-warp register-resident sparse kernel (H > 512): one sequence of at most 40 steps
+    computes its projection inside the recurrent launch (two launches for two layers), a longer one does not;
+    both directions, a ragged last timestep tile, non-zero initial state."""
+    import torch
+    import paper_1901_10997_b200 as pkg
+    monkeypatch.delenv("LSTM_B200_PROJ", raising=False)
+    monkeypatch.delenv("LSTM_B200_FUSE", raising=False)
+    w = small("csr_fused", 2, True, 90, 600, T, 1, "bf16", scale=0.15, density=0.1, seed=9)
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    m = pkg.LSTM(csr_weights(oracle, weights), layers=2, in_dim=w.in_dim, hidden=w.hidden, bidir=True, dtype="bf16",
+                 exec_mode="csr", max_T=T, max_B=1)
+    try:
+        assert m.info()["recur_csr_register_resident"] == 1
+        y, hT, cT = m.forward(torch.from_numpy(x).cuda(), torch.from_numpy(h0).cuda(), torch.from_numpy(c0).cuda())
+        m.check()
+        assert m.info()["launches_per_forward"] == (2 if fused else 5)
+        assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"{w.name}/T={T}")
+    finally:
+        m.close()
