@@ -374,7 +374,7 @@ int max_b_fits(const lstm_handle *h)
 // Operand-A fragments of a [4U x K] matrix whose row q*U + u is gate q of unit u: per CTA (units split
 // evenly over ncta CTAs) [warp][column tile][row tile][lane] x 4 words, local row = 4 * unit + gate,
 // zero beyond the CTA's units and beyond column K.
-std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int NW, int nkw, int MT)
+std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int NW, int nkw, int MT, bool adjacent = false)
 {
     std::vector<uint32_t> f((size_t)ncta * NW * nkw * MT * 32 * 4, 0u);
     size_t o = 0;
@@ -390,7 +390,9 @@ std::vector<uint32_t> pack_fragments(const float *m, int U, int K, int ncta, int
                     for (int lane = 0; lane < 32; ++lane) {
                         const int g = lane >> 2, p2 = (lane & 3) * 2;
                         const int r0 = mt * 16 + g, r1 = r0 + 8;
-                        const int ka = (wp * nkw + i) * 16 + p2, kb = ka + 8;
+                        // adjacent: the lane's four MMA k slots hold the adjacent columns 4 * (lane & 3) .. + 3 (the
+                        // input-projection fragments, whose other operand is then one 16-byte load)
+                        const int ka = (wp * nkw + i) * 16 + (adjacent ? 2 * p2 : p2), kb = adjacent ? ka + 2 : ka + 8;
                         f[o++] = wv(r0, ka) | (wv(r0, ka + 1) << 16);
                         f[o++] = wv(r1, ka) | (wv(r1, ka + 1) << 16);
                         f[o++] = wv(r0, kb) | (wv(r0, kb + 1) << 16);
@@ -644,7 +646,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                     // recurrent kernel's prologue
                     const int nranges = h->mma_nw / 2;                 // two warps share a column range
                     ly.nkw_x = ((ly.in_l + 15) / 16 + nranges - 1) / nranges;
-                    const std::vector<uint32_t> fx = pack_fragments(m.data(), H, ly.in_l, h->ncta_dir, nranges, ly.nkw_x, h->mma_mt);
+                    const std::vector<uint32_t> fx = pack_fragments(m.data(), H, ly.in_l, h->ncta_dir, nranges, ly.nkw_x, h->mma_mt, true);
                     rc = upload(h, (uint32_t **)&ly.xfrag[d], fx.data(), fx.size() * 4, st, "input weight fragments");
                     if (rc == LSTM_OK) cudaStreamSynchronize(st);
                     if (rc) break;
@@ -739,7 +741,7 @@ static int create_impl(lstm_handle **out, int layers, int in_dim, int hidden, in
                         for (int e = cx.rowptr[r]; e < cx.rowptr[r + 1]; ++e) m[(size_t)r * ly.in_l + cx.col[e]] = cx.val[e];
                     const int nranges = h->csr_nw / 2;
                     ly.nkw_x = ((ly.in_l + 15) / 16 + nranges - 1) / nranges;
-                    const std::vector<uint32_t> fx = pack_fragments(m.data(), H, ly.in_l, h->ncta_dir, nranges, ly.nkw_x, h->csr_mt);
+                    const std::vector<uint32_t> fx = pack_fragments(m.data(), H, ly.in_l, h->ncta_dir, nranges, ly.nkw_x, h->csr_mt, true);
                     rc = upload(h, (uint32_t **)&ly.xfrag[d], fx.data(), fx.size() * 4, st, "input weight fragments");
                     if (rc == LSTM_OK) cudaStreamSynchronize(st);
                     if (rc) break;

@@ -131,7 +131,8 @@ __device__ __forceinline__ void finish_unit(const FinishLane &f, const float *re
 // Input projection inside a recurrent kernel's prologue (single sequence of at most kFuseMaxT steps): the CTA's
 // own rows of G = X Wx^T + b for every timestep, left in shared memory as [kFuseMaxT][MT * 16 + 1] floats at
 // byte offset gs_off.  Wx arrives as mma.sync operand-A fragments (xfrag_d: this direction's, laid out
-// [cta][NW / 2 column ranges][nkx 16-column tiles][MT][32 lanes] uint4); the activations are split into bf16 hi
+// [cta][NW / 2 column ranges][nkx 16-column tiles][MT][32 lanes] uint4, the columns inside a tile permuted as
+// described at the loads below); the activations are split into bf16 hi
 // and lo terms on the fly.  Work split: the NW / 2 column ranges are each taken by two warps, one for the first
 // 24 timesteps and one for the rest, so that the accumulators of a warp stay few and two loads can be in flight.
 // Every warp leaves its partial products in its own block at the start of shared memory (NW * 24 * (MT * 16 + 1)
@@ -160,18 +161,24 @@ __device__ __forceinline__ float *fused_projection(unsigned char *smem, size_t g
     const int t0 = half * NTH * 8;
     uint4 af[MT], an[MT];
     float xv[NTH][4], xn[NTH][4];
+    const bool vec = (in_l & 3) == 0 && (reinterpret_cast<size_t>(X) & 15) == 0;     // rows of X start on 16 bytes
     auto fetch = [&](int i, uint4 (&fa)[MT], float (&fx)[NTH][4]) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) fa[mt] = i < nkx ? __ldg(xsrc + (size_t)(i * MT + mt) * 32) : make_uint4(0, 0, 0, 0);
-        const int k0 = (range * nkx + i) * 16 + 2 * tig;
+        // The fragments are packed with the columns of a 16-wide tile permuted so that the four a lane multiplies
+        // (MMA k slots 2 tig, 2 tig + 1, 2 tig + 8, 2 tig + 9) are the adjacent columns 4 tig .. 4 tig + 3: one
+        // 16-byte load per (lane, timestep tile) where the rows of X allow it, four scalar loads otherwise.
+        const int k0 = (range * nkx + i) * 16 + 4 * tig;
 #pragma unroll
         for (int nt = 0; nt < NTH; ++nt) {
             const int t = t0 + nt * 8 + g;
             const float *xr = X + (size_t)t * in_l;
+            if (vec && i < nkx && t < T && k0 + 3 < in_l) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(xr + k0));
+                fx[nt][0] = v.x; fx[nt][1] = v.y; fx[nt][2] = v.z; fx[nt][3] = v.w;
+            } else {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int k = k0 + (e & 1) + (e >> 1) * 8;
-                fx[nt][e] = (i < nkx && t < T && k < in_l) ? __ldg(xr + k) : 0.0f;
+                for (int e = 0; e < 4; ++e) fx[nt][e] = (i < nkx && t < T && k0 + e < in_l) ? __ldg(xr + k0 + e) : 0.0f;
             }
         }
     };
