@@ -113,3 +113,35 @@ def test_sparse_kernel_projects_in_its_prologue_for_short_single_sequences(oracl
         assert_close((y.cpu().numpy(), hT.cpu().numpy(), cT.cpu().numpy()), ref, "bf16", f"{w.name}/T={T}")
     finally:
         m.close()
+
+
+def _random_cases(n, seed):
+    """Shapes nobody picked by hand for the paths added last: sparse and dense single sequences around the 40-step
+    limit of the fused prologue, and batches whose T*B spans several activation tiles of the projection."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        kind = ["csr1", "dense1", "projbig"][i % 3]
+        L, bidir = int(rng.integers(1, 3)), bool(rng.integers(0, 2))
+        if kind == "csr1":
+            c = dict(H=int(rng.integers(520, 1500)), B=int(rng.integers(1, 4)), T=int(rng.integers(1, 45)), in_dim=int(rng.integers(1, 300)),
+                     mode="csr", density=float(rng.choice([0.05, 0.1, 0.3])))
+        elif kind == "dense1":
+            c = dict(H=int(rng.integers(100, 1600)), B=1, T=int(rng.integers(1, 45)), in_dim=int(rng.integers(1, 400)), mode="dense", density=1.0)
+        else:
+            c = dict(H=int(rng.integers(30, 500)), B=int(rng.integers(8, 40)), T=int(rng.integers(6, 30)), in_dim=int(rng.integers(8, 300)),
+                     mode="dense", density=1.0)
+        cases.append(dict(c, kind=kind, L=L, bidir=bidir, seed=7000 + i))
+    return cases
+
+
+@pytest.mark.parametrize("c", _random_cases(24, 31), ids=lambda c: "{kind}_L{L}D{d}_in{in_dim}_H{H}_T{T}_B{B}".format(d=1 + c["bidir"], **c))
+def test_random_shapes_of_the_fused_and_large_projection_paths(oracle, c):
+    import paper_1901_10997_b200 as pkg
+    scale = min(0.3, 2.0 / np.sqrt(c["H"] + c["in_dim"]))
+    w = wl.Workload("rnd", c["L"], c["bidir"], c["in_dim"], c["H"], c["T"], c["B"], "bf16", scale, density=c["density"], seed=c["seed"])
+    weights, x = wl.make(w)
+    h0, c0 = wl.make_states(w)
+    ref = oracle.forward(weights, x, h0, c0, layers=w.layers, bidir=w.bidir, hidden=w.hidden)
+    got, _ = _forward(pkg, w, weights if c["mode"] == "dense" else csr_weights(oracle, weights), x, h0, c0, exec_mode=c["mode"])
+    assert_close(got, ref, "bf16", "rnd/" + c["kind"])
